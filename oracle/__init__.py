@@ -1,0 +1,17 @@
+"""CPU oracle for BalanceKV -- test infrastructure only.
+
+Only tests, the smoke check and the bench's CPU baseline may import this package;
+the CUDA library and its Python binding never do.
+"""
+from .binding import (  # noqa: F401
+    OracleParams,
+    OracleStream,
+    build,
+    compress_streams,
+    num_threads,
+    philox4x32_10,
+    softmax_balance,
+    walk_constant,
+    walk_uniform,
+    weighted_attention,
+)
