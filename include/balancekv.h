@@ -1,0 +1,160 @@
+/*
+ * balancekv.h -- C ABI of the BalanceKV hot path on NVIDIA B200 (sm_100a).
+ *
+ * BalanceKV ("Streaming Attention Approximation via Discrepancy Theory") compresses the
+ * key/value cache of every (sequence, layer, KV head) stream: batches of t tokens are
+ * halved by SoftmaxBalance (Algorithm 2: a self-balancing walk over the pairwise kernel
+ * exp(<k_i,k_j>/sqrt d) <v_i,v_j>), survivors double their weight and climb the
+ * MergeAndReduce tree (Algorithm 3) up to level T, and decode attention is the ratio of
+ * Algorithm 1's output step evaluated over the weighted sets C^0..C^T (Theorem 3.3's
+ * estimator) -- here over one shared set for numerator and denominator.
+ *
+ * Conventions
+ *   - Every call returns 0 (BALANCEKV_OK) or a negative error code; nothing throws.
+ *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by the
+ *     caller, row-major and contiguous.  The library copies what it keeps and never
+ *     frees or retains caller memory.
+ *   - Work is enqueued asynchronously on the CUDA stream passed as `stream`
+ *     (a cudaStream_t cast to void*; NULL = the default stream).  A context must be used
+ *     from one host thread at a time, on the device that was current at create time.
+ *   - dtype: 0 = float32, 1 = bfloat16 (keys, values, queries and outputs alike).
+ *   - A "stream" below is one (sequence, layer, KV head) token stream of the paper's
+ *     streaming formulation (Section 2.1); `stream` (void*) is the CUDA stream.
+ *   - There is no CPU fallback: without a CUDA device every device call fails with
+ *     BALANCEKV_E_CUDA.
+ */
+#ifndef BALANCEKV_H_
+#define BALANCEKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BALANCEKV_OK 0
+#define BALANCEKV_E_INVAL (-1)   /* bad argument, shape, dtype or state                 */
+#define BALANCEKV_E_NOMEM (-2)   /* a stream's capacity (or device memory) is exhausted */
+#define BALANCEKV_E_STATE (-3)   /* call not valid in the context's current state       */
+#define BALANCEKV_E_CUDA (-4)    /* a CUDA runtime call failed                          */
+#define BALANCEKV_E_TIMEOUT (-5) /* a bounded device-side wait gave up                  */
+
+typedef struct balancekv_ctx balancekv_ctx;
+
+/* Parameters of Algorithms 1-3 (r, t, T, delta) plus the shape of the model. */
+typedef struct balancekv_config {
+  int32_t n_seqs;        /* B: sequences                                                      */
+  int32_t n_layers;      /* L                                                                 */
+  int32_t n_kv_heads;    /* H                                                                 */
+  int32_t n_q_heads;     /* H*g, g = query heads per KV head (1..8)                           */
+  int32_t head_dim;      /* d: 64 or 128                                                      */
+  int32_t dtype;         /* 0 = float32, 1 = bfloat16                                         */
+  int32_t block;         /* t: batch size of Algorithm 3 = tokens per SoftmaxBalance call;
+                            multiple of 64                                                    */
+  int32_t levels;        /* T >= 0: compression rate 2^-T; 0 keeps every token                */
+  int32_t max_tokens;    /* N: most tokens a stream will ever receive; also delta's default   */
+  int32_t max_pending;   /* most tokens appended to a stream between two compress calls;
+                            <= 0 means N (always safe)                                        */
+  int32_t recent_window; /* W >= 0: the newest W tokens of a stream never enter a call        */
+  int32_t center_keys;   /* 1: subtract the call's mean key inside the kernel only
+                            (the stored keys are untouched); 0 (default): off                 */
+  int32_t gram_path;     /* 0 = automatic, 1 = CUDA-core (fp32 FMA) kernel, 2 = tensor-core
+                            (tcgen05) kernel; 2 needs bf16, d = 128, t multiple of 128        */
+  int32_t reserved;
+  uint64_t seed;         /* Philox key; sequence s uses seed + s                              */
+  float delta;           /* failure probability of Algorithm 2; <= 0 means 1/N^2              */
+  float c_override;      /* > 0: use this c instead of 30 ln(t/delta)                         */
+  float r_key, r_value;  /* > 0: fixed radii of Algorithm 2; <= 0: per-call maxima            */
+} balancekv_config;
+
+typedef struct balancekv_stats_t {
+  int64_t tokens_appended;    /* over all streams                                             */
+  int64_t tokens_stored;      /* rows currently held (all levels, all streams)                */
+  int64_t calls_run;          /* SoftmaxBalance calls executed                                */
+  int64_t walk_fails;         /* times |y^T eta| exceeded c R^2 (counted, clamped, no error)  */
+  int64_t device_status;      /* 0, or the first device-side error code                       */
+  int64_t bytes_resident;     /* device memory owned by the context                           */
+  int64_t kernels_launched;   /* kernels of this library launched so far                      */
+} balancekv_stats_t;
+
+/* Allocate a context: all cache memory for n_seqs*n_layers*n_kv_heads streams.
+ * E_INVAL on a bad field, E_NOMEM / E_CUDA if the device allocation fails. */
+int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out);
+int balancekv_destroy(balancekv_ctx* ctx);
+
+/* Algorithm 3, "C^0 <- C^0 + {k_j, v_j}": append n_tokens rows to one stream.
+ * K_blk, V_blk: [n_tokens, head_dim].  No compression work happens here.
+ * E_NOMEM if the stream would exceed max_tokens or its pending capacity. */
+int balancekv_stream_append(balancekv_ctx* ctx, int seq, int layer, int kv_head, const void* K_blk,
+                            const void* V_blk, int n_tokens, void* stream);
+
+/* Same for every stream of one layer at once.
+ * K, V: [n_seqs, n_kv_heads, n_tokens, head_dim]. */
+int balancekv_stream_append_layer(balancekv_ctx* ctx, int layer, const void* K, const void* V,
+                                  int n_tokens, void* stream);
+
+/* As above with HOST buffers (pinned memory recommended): the copy to the device is
+ * enqueued on `stream` through a staging buffer owned by the context, which the next
+ * *_host call reuses (such calls must all be issued on the same CUDA stream). */
+int balancekv_stream_append_layer_host(balancekv_ctx* ctx, int layer, const void* K_host,
+                                       const void* V_host, int n_tokens, void* stream);
+
+/* Algorithm 3's update step for every stream: run every SoftmaxBalance call that is ready
+ * (a full batch of t eligible tokens in C^0, or two halves in C^i, i < T), level by level,
+ * including the strict-half selection of the paper's implementation note (Appendix B).
+ * T must equal config.levels (E_INVAL otherwise); T = 0 is a no-op. */
+int balancekv_compress(balancekv_ctx* ctx, int T, void* stream);
+/* Same, restricted to the streams of one layer. */
+int balancekv_compress_layer(balancekv_ctx* ctx, int layer, int T, void* stream);
+
+/* Algorithm 1's output ratio / Theorem 3.3's estimator for one layer:
+ * out[s,h,:] = sum_i w_i e^{<k_i,q>/sqrt d} v_i / sum_i w_i e^{<k_i,q>/sqrt d} over every
+ * stored token of the stream of (s, h / g), w_i = 2^level.  q, out: [n_seqs, n_q_heads,
+ * head_dim] in the context's dtype.  With T = 0 this is Eq. (1) exactly. */
+int balancekv_decode_attn(balancekv_ctx* ctx, int layer, const void* q, void* out, void* stream);
+
+/* As above with HOST q and out: q is copied in, out copied back, both on `stream`;
+ * the call returns without synchronising (synchronise the stream before reading out). */
+int balancekv_decode_attn_host(balancekv_ctx* ctx, int layer, const void* q_host, void* out_host,
+                               void* stream);
+
+/* Load an already-compressed set into level `level` of every stream of one layer
+ * (weight 2^level, the weights of Theorem 3.3's estimator): K, V: [n_seqs, n_kv_heads,
+ * n_tokens, head_dim]; orig_idx (may be NULL): [n_seqs, n_kv_heads, n_tokens] original
+ * token positions.  level in [0, T]; for 1 <= level < T at most t rows fit. */
+int balancekv_cache_load_level(balancekv_ctx* ctx, int layer, int level, const void* K, const void* V,
+                               const int32_t* orig_idx, int n_tokens, void* stream);
+
+/* Inspection.  Gathers the stream's weighted set in the order C^T, ..., C^1, C^0
+ * (ascending original position) into buffers owned by the context and returns DEVICE
+ * pointers to them, valid until the next call on the context.  Synchronises the device.
+ * Any output pointer may be NULL. */
+int balancekv_cache_view(balancekv_ctx* ctx, int seq, int layer, int kv_head, const void** K,
+                         const void** V, const float** w, const int32_t** orig_idx, int* len);
+
+/* Host-side bookkeeping of one stream: sizes_host[0..T] = |C^0| .. |C^T| (Algorithm 3). */
+int balancekv_level_sizes(balancekv_ctx* ctx, int seq, int layer, int kv_head, int32_t* sizes_host);
+
+/* Record, for every later call, the signs eta, the running correlation
+ * S_j = y^T eta / R^2 and the probability p_j of Algorithm 2.  Allocates the record
+ * buffers; must be enabled before the first compress. */
+int balancekv_debug_enable(balancekv_ctx* ctx, int on);
+/* DEVICE pointers to the record of call (level, ordinal) of a stream, each [t]. */
+int balancekv_debug_call(balancekv_ctx* ctx, int seq, int layer, int kv_head, int level,
+                         int call_ordinal, const int8_t** eta, const float** S, const float** p,
+                         int* m);
+
+int balancekv_stats(balancekv_ctx* ctx, balancekv_stats_t* out);
+const char* balancekv_strerror(int code);
+
+/* Pure host bookkeeping of Algorithm 3 (no device needed): a stream holds
+ * appended_after_event[e] tokens after its e-th append, and compress runs after every
+ * append; writes the calls that fire, in launch order, as (event, level, ordinal)
+ * triples.  Returns the number of calls (at most max_calls are written) or an error. */
+int balancekv_plan_calls(int block, int levels, int recent_window, const int32_t* appended_after_event,
+                         int n_events, int32_t* calls_out, int max_calls);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BALANCEKV_H_ */

@@ -1,1 +1,10 @@
 """BalanceKV hot path on B200: C-ABI CUDA library plus a thin ctypes binding."""
+from .binding import (  # noqa: E402,F401
+    BalanceKVError,
+    Config,
+    Context,
+    EXPORTS,
+    LIB_PATH,
+    load,
+    plan_calls,
+)

@@ -1,0 +1,673 @@
+// C ABI of the BalanceKV library: context, memory layout, launch scheduling.
+// Every step of the hot path runs in the CUDA kernels of this directory; this file only
+// validates arguments, keeps Algorithm 3's bookkeeping (sched.h) and enqueues launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/balancekv.h"
+#include "common.cuh"
+#include "sched.h"
+
+using namespace bkv;
+
+namespace bkv {
+bool walk_tc_supported(const Geom& G);
+cudaError_t walk_tc_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** tmaps_out);
+void walk_tc_release(void* tmaps);
+}  // namespace bkv
+
+#define BKV_CUDA(expr)                                                                    \
+  do {                                                                                    \
+    cudaError_t _e = (expr);                                                              \
+    if (_e != cudaSuccess) {                                                              \
+      std::fprintf(stderr, "balancekv: %s failed: %s (%s:%d)\n", #expr, cudaGetErrorString(_e), \
+                   __FILE__, __LINE__);                                                   \
+      return _e == cudaErrorMemoryAllocation ? BALANCEKV_E_NOMEM : BALANCEKV_E_CUDA;      \
+    }                                                                                     \
+  } while (0)
+
+struct balancekv_ctx {
+  balancekv_config cfg{};
+  Geom G{};
+  Layout Lo{};
+  Arena A{};
+  int n_streams = 0, device = 0, sm_count = 148;
+  int64_t total_rows = 0;
+  std::vector<StreamState> st;
+  size_t bytes_resident = 0;
+  int esz = 2;
+
+  // per-launch buffers
+  int max_calls = 0;
+  CallStat* d_stats = nullptr;
+  float* d_tokshift = nullptr;
+  int8_t* d_eta = nullptr;
+  unsigned long long* d_fail = nullptr;
+  int* d_status = nullptr;
+  float* d_decode_scratch = nullptr;
+  int max_splits = 1;
+  bool use_tc = false;
+  void* tmaps = nullptr;
+
+  // descriptor ring: two halves of pinned host memory mirrored on the device
+  char* h_ring = nullptr;
+  char* d_ring = nullptr;
+  size_t ring_half = 0, ring_pos = 0;
+  int ring_cur = 0;
+  cudaEvent_t ring_ev[2]{};
+  bool ring_ev_valid[2] = {false, false};
+
+  // debug records
+  bool debug = false;
+  int8_t* dbg_eta = nullptr;
+  float* dbg_S = nullptr;
+  float* dbg_p = nullptr;
+  int64_t dbg_calls_per_stream = 0;
+  int64_t dbg_level_base[kMaxLevels + 1] = {};
+
+  // inspection view
+  void* view_K = nullptr;
+  void* view_V = nullptr;
+  float* view_w = nullptr;
+  int32_t* view_idx = nullptr;
+  int64_t view_cap = 0;
+
+  // staging for the *_host entry points
+  void* bounce_K = nullptr;
+  void* bounce_V = nullptr;
+  size_t bounce_bytes = 0;
+  void* bounce_q = nullptr;
+  void* bounce_out = nullptr;
+
+  int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(balancekv_ctx* c, T** p, size_t count) {
+  const size_t bytes = std::max<size_t>(count * sizeof(T), 256);
+  BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(p), bytes));
+  c->bytes_resident += bytes;
+  return BALANCEKV_OK;
+}
+
+// Copies a host array into the descriptor ring and returns its device address.
+int ring_push(balancekv_ctx* c, const void* data, size_t bytes, cudaStream_t st, void** dev) {
+  const size_t need = (bytes + 255) & ~(size_t)255;
+  if (need > c->ring_half) return BALANCEKV_E_NOMEM;
+  if (c->ring_pos + need > c->ring_half) {
+    BKV_CUDA(cudaEventRecord(c->ring_ev[c->ring_cur], st));
+    c->ring_ev_valid[c->ring_cur] = true;
+    c->ring_cur ^= 1;
+    c->ring_pos = 0;
+    if (c->ring_ev_valid[c->ring_cur]) BKV_CUDA(cudaEventSynchronize(c->ring_ev[c->ring_cur]));
+  }
+  const size_t off = (size_t)c->ring_cur * c->ring_half + c->ring_pos;
+  std::memcpy(c->h_ring + off, data, bytes);
+  BKV_CUDA(cudaMemcpyAsync(c->d_ring + off, c->h_ring + off, bytes, cudaMemcpyHostToDevice, st));
+  c->ring_pos += need;
+  *dev = c->d_ring + off;
+  return BALANCEKV_OK;
+}
+
+int stream_id(const balancekv_ctx* c, int seq, int layer, int head) {
+  return (seq * c->cfg.n_layers + layer) * c->cfg.n_kv_heads + head;
+}
+
+int64_t dbg_offset(const balancekv_ctx* c, int stream, int level, int64_t ordinal) {
+  return ((int64_t)stream * c->dbg_calls_per_stream + c->dbg_level_base[level] + ordinal) * c->cfg.block;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_config(const balancekv_config& f) {
+  if (f.n_seqs < 1 || f.n_layers < 1 || f.n_kv_heads < 1 || f.n_q_heads < 1) return BALANCEKV_E_INVAL;
+  if (f.n_layers > 65535 || f.n_kv_heads > 65535) return BALANCEKV_E_INVAL;
+  if (f.n_q_heads % f.n_kv_heads) return BALANCEKV_E_INVAL;
+  const int g = f.n_q_heads / f.n_kv_heads;
+  if (g < 1 || g > kMaxGroup) return BALANCEKV_E_INVAL;
+  if (f.head_dim != 64 && f.head_dim != 128) return BALANCEKV_E_INVAL;
+  if (f.dtype != 0 && f.dtype != 1) return BALANCEKV_E_INVAL;
+  if (f.block < 64 || f.block % 64 || f.block > 4096) return BALANCEKV_E_INVAL;
+  if (f.levels < 0 || f.levels > kMaxLevels) return BALANCEKV_E_INVAL;
+  if (f.max_tokens < 1 || f.recent_window < 0) return BALANCEKV_E_INVAL;
+  if (f.gram_path < 0 || f.gram_path > 2) return BALANCEKV_E_INVAL;
+  return BALANCEKV_OK;
+}
+
+// Builds the per-stream region layout (rows) for the given parameters.
+void build_layout(const balancekv_config& f, int max_pending, Layout& Lo) {
+  const int t = f.block, T = f.levels, N = f.max_tokens;
+  Lo.t = t; Lo.T = T; Lo.W = f.recent_window;
+  if (T == 0) {
+    Lo.cap0 = N; Lo.capT = 0;
+    Lo.region_off[0] = 0;
+    Lo.R = N;
+    return;
+  }
+  const int64_t calls_top = (int64_t)N / ((int64_t)t << (T - 1));
+  Lo.capT = (int32_t)std::max<int64_t>(calls_top * (t / 2), ((int64_t)N + (1 << T) - 1) >> T);
+  Lo.cap0 = (int32_t)std::min<int64_t>((int64_t)max_pending + 2 * ((int64_t)t + f.recent_window),
+                                       (int64_t)N + 2 * ((int64_t)t + f.recent_window));
+  int64_t off = 0;
+  Lo.region_off[T] = (int32_t)off; off += Lo.capT;
+  for (int l = T - 1; l >= 1; --l) { Lo.region_off[l] = (int32_t)off; off += 2 * t; }
+  Lo.region_off[0] = (int32_t)off; off += Lo.cap0;
+  Lo.R = (off + 63) / 64 * 64;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* balancekv_strerror(int code) {
+  switch (code) {
+    case BALANCEKV_OK: return "ok";
+    case BALANCEKV_E_INVAL: return "invalid argument";
+    case BALANCEKV_E_NOMEM: return "capacity or memory exhausted";
+    case BALANCEKV_E_STATE: return "call not valid in the current state";
+    case BALANCEKV_E_CUDA: return "CUDA runtime error";
+    case BALANCEKV_E_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown error";
+}
+
+int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
+  if (!cfg || !out) return BALANCEKV_E_INVAL;
+  *out = nullptr;
+  int rc = check_config(*cfg);
+  if (rc) return rc;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return BALANCEKV_E_CUDA;
+  balancekv_ctx* c = new (std::nothrow) balancekv_ctx();
+  if (!c) return BALANCEKV_E_NOMEM;
+  c->cfg = *cfg;
+  const balancekv_config& f = c->cfg;
+  BKV_CUDA(cudaGetDevice(&c->device));
+  BKV_CUDA(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
+  c->esz = f.dtype ? 2 : 4;
+  const int t = f.block, T = f.levels, N = f.max_tokens;
+  const int max_pending = f.max_pending > 0 ? std::min(f.max_pending, N) : N;
+  build_layout(f, max_pending, c->Lo);
+  c->n_streams = f.n_seqs * f.n_layers * f.n_kv_heads;
+  c->st.assign(c->n_streams, StreamState());
+
+  // most level-0 calls of one batched launch, and the ping-pong pools behind the streams
+  const size_t row_bytes = (size_t)f.head_dim * c->esz;
+  if (T > 0) {
+    const size_t per_call = (size_t)(t / 2) * row_bytes * 2;          // K+V survivors of one call
+    const size_t budget = (size_t)256 << 20;                          // both pools together
+    int64_t mc = (int64_t)(budget / (2 * per_call));
+    mc = std::max<int64_t>(2, std::min<int64_t>(mc, 4096));
+    c->max_calls = (int)mc;
+    c->Lo.pool_pairs = T > 1 ? (mc + 1) / 2 : 0;
+  }
+  const int64_t stream_rows = (int64_t)c->n_streams * c->Lo.R;
+  c->Lo.pool_row[0] = stream_rows;
+  c->Lo.pool_row[1] = stream_rows + c->Lo.pool_pairs * t;
+  c->total_rows = stream_rows + 2 * c->Lo.pool_pairs * t;
+
+  Geom& G = c->G;
+  G.d = f.head_dim; G.t = t; G.T = T; G.H = f.n_kv_heads; G.L = f.n_layers; G.B = f.n_seqs;
+  G.g = f.n_q_heads / f.n_kv_heads;
+  G.is_bf16 = f.dtype;
+  G.rows_per_stream = c->Lo.R;
+  for (int l = 0; l <= kMaxLevels; ++l) G.region_off[l] = c->Lo.region_off[l];
+  G.inv_sqrt_d = (float)(1.0 / std::sqrt((double)f.head_dim));
+  {
+    // c = 30 log(n/delta), natural log, n = tokens of a call, delta = 1/N^2 by default
+    const double delta = f.delta > 0 ? (double)f.delta : 1.0 / ((double)N * (double)N);
+    const double cc = f.c_override > 0 ? (double)f.c_override : 30.0 * std::log((double)t / delta);
+    G.c = (float)cc;
+  }
+  G.fixed_rk2 = f.r_key > 0 ? (float)((double)f.r_key * f.r_key) : 0.f;
+  G.fixed_rv2 = f.r_value > 0 ? (float)((double)f.r_value * f.r_value) : 0.f;
+  G.seed = f.seed;
+  G.center_keys = f.center_keys ? 1 : 0;
+
+  auto fail = [&](int code) { balancekv_destroy(c); return code; };
+  if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->A.K), (size_t)c->total_rows * row_bytes))) return fail(rc);
+  if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->A.V), (size_t)c->total_rows * row_bytes))) return fail(rc);
+  if ((rc = dev_alloc(c, &c->A.idx, (size_t)c->total_rows))) return fail(rc);
+  if ((rc = dev_alloc(c, &c->A.seg, (size_t)c->n_streams * (T + 1)))) return fail(rc);
+  if (cudaMemset(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (T + 1)) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  if (T > 0) {
+    if ((rc = dev_alloc(c, &c->d_stats, (size_t)c->max_calls))) return fail(rc);
+    if ((rc = dev_alloc(c, &c->d_eta, (size_t)c->max_calls * t))) return fail(rc);
+    if (G.center_keys && (rc = dev_alloc(c, &c->d_tokshift, (size_t)c->max_calls * (t + f.head_dim)))) return fail(rc);
+  }
+  if ((rc = dev_alloc(c, &c->d_fail, 1))) return fail(rc);
+  if ((rc = dev_alloc(c, &c->d_status, 1))) return fail(rc);
+  if (cudaMemset(c->d_fail, 0, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  {
+    const int n_sl = f.n_seqs * f.n_kv_heads;
+    c->max_splits = std::max(1, std::min(64, (2 * c->sm_count + n_sl - 1) / n_sl));
+    const size_t sb = decode_scratch_bytes(G, c->max_splits);
+    if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->d_decode_scratch), sb))) return fail(rc);
+    if (cudaMemset(c->d_decode_scratch, 0, sb) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  }
+  c->ring_half = (size_t)4 << 20;
+  if (cudaMallocHost(reinterpret_cast<void**>(&c->h_ring), 2 * c->ring_half) != cudaSuccess) return fail(BALANCEKV_E_NOMEM);
+  if ((rc = dev_alloc(c, &c->d_ring, 2 * c->ring_half))) return fail(rc);
+  for (int i = 0; i < 2; ++i)
+    if (cudaEventCreateWithFlags(&c->ring_ev[i], cudaEventDisableTiming) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+
+  const bool tc_ok = walk_tc_supported(G) && c->total_rows < ((int64_t)1 << 31);
+  if (f.gram_path == 2 && !tc_ok) return fail(BALANCEKV_E_INVAL);
+  c->use_tc = T > 0 && tc_ok && f.gram_path != 1;
+  if (c->use_tc) {
+    if (walk_tc_prepare(G, c->A, c->total_rows, &c->tmaps) != cudaSuccess) {
+      if (f.gram_path == 2) return fail(BALANCEKV_E_CUDA);
+      c->use_tc = false;
+    }
+  }
+  if (T > 0 && !c->use_tc) {
+    if (!walk_simt_supported(G.d)) return fail(BALANCEKV_E_INVAL);
+    if (walk_simt_smem_bytes(G.d, t) > (size_t)227 * 1024) return fail(BALANCEKV_E_INVAL);
+  }
+  *out = c;
+  return BALANCEKV_OK;
+}
+
+int balancekv_destroy(balancekv_ctx* c) {
+  if (!c) return BALANCEKV_E_INVAL;
+  cudaDeviceSynchronize();
+  walk_tc_release(c->tmaps);
+  void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
+                  c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
+                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  if (c->h_ring) cudaFreeHost(c->h_ring);
+  for (int i = 0; i < 2; ++i)
+    if (c->ring_ev[i]) cudaEventDestroy(c->ring_ev[i]);
+  delete c;
+  return BALANCEKV_OK;
+}
+
+// Appends (level 0) or loads (level T) n rows per listed stream from a caller tensor laid
+// out as consecutive [n, d] blocks in the order of `streams`.
+static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int level, const void* K, const void* V,
+                       const int32_t* idx, int n, cudaStream_t st) {
+  if (!K || !V || n < 0) return BALANCEKV_E_INVAL;
+  if (!aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
+  if (n == 0) return BALANCEKV_OK;
+  const balancekv_config& f = c->cfg;
+  const Layout& Lo = c->Lo;
+  const int T = Lo.T;
+  const int max_pending = T == 0 ? f.max_tokens : (f.max_pending > 0 ? std::min(f.max_pending, f.max_tokens) : f.max_tokens);
+  for (int s : streams) {
+    const StreamState& S = c->st[s];
+    if (level == 0) {
+      if (S.appended + n > f.max_tokens) return BALANCEKV_E_NOMEM;
+      if (S.pending + n > max_pending) return BALANCEKV_E_NOMEM;
+      if ((int64_t)S.start0 + S.len0 + n > Lo.cap0) return BALANCEKV_E_NOMEM;
+    } else {
+      if ((int64_t)S.lvl_len[T] + n > Lo.capT) return BALANCEKV_E_NOMEM;
+    }
+  }
+  std::vector<AppendDesc> descs(streams.size());
+  for (size_t i = 0; i < streams.size(); ++i) {
+    const int s = streams[i];
+    StreamState& S = c->st[s];
+    AppendDesc& D = descs[i];
+    D.src_off = (int64_t)i * n * f.head_dim;
+    D.stream = s; D.n = n; D.level = level; D.pad = 0;
+    if (level == 0) {
+      D.dst_row = (int64_t)s * Lo.R + Lo.region_off[0] + S.start0 + S.len0;
+      D.idx0 = (int32_t)S.appended;
+      S.len0 += n; S.appended += n; S.pending += n;
+      D.new_len = S.len0;
+      c->tokens_appended += n;
+    } else {
+      D.dst_row = (int64_t)s * Lo.R + Lo.region_off[T] + S.lvl_len[T];
+      D.idx0 = S.lvl_len[T];
+      S.lvl_len[T] += n;
+      D.new_len = S.lvl_len[T];
+    }
+  }
+  void* d_descs = nullptr;
+  int rc = ring_push(c, descs.data(), descs.size() * sizeof(AppendDesc), st, &d_descs);
+  if (rc) return rc;
+  BKV_CUDA(launch_append(c->G, c->A, static_cast<const AppendDesc*>(d_descs), (int)descs.size(), n, K, V, idx, st));
+  c->kernels_launched++;
+  return BALANCEKV_OK;
+}
+
+int balancekv_stream_append(balancekv_ctx* c, int seq, int layer, int kv_head, const void* K_blk, const void* V_blk,
+                            int n_tokens, void* stream) {
+  if (!c) return BALANCEKV_E_INVAL;
+  const balancekv_config& f = c->cfg;
+  if (seq < 0 || seq >= f.n_seqs || layer < 0 || layer >= f.n_layers || kv_head < 0 || kv_head >= f.n_kv_heads)
+    return BALANCEKV_E_INVAL;
+  std::vector<int> s{stream_id(c, seq, layer, kv_head)};
+  return append_impl(c, s, 0, K_blk, V_blk, nullptr, n_tokens, static_cast<cudaStream_t>(stream));
+}
+
+static std::vector<int> layer_streams(const balancekv_ctx* c, int layer) {
+  std::vector<int> v;
+  for (int s = 0; s < c->cfg.n_seqs; ++s)
+    for (int h = 0; h < c->cfg.n_kv_heads; ++h) v.push_back(stream_id(c, s, layer, h));
+  return v;
+}
+
+int balancekv_stream_append_layer(balancekv_ctx* c, int layer, const void* K, const void* V, int n_tokens, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
+  return append_impl(c, layer_streams(c, layer), 0, K, V, nullptr, n_tokens, static_cast<cudaStream_t>(stream));
+}
+
+int balancekv_stream_append_layer_host(balancekv_ctx* c, int layer, const void* K_host, const void* V_host,
+                                       int n_tokens, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !K_host || !V_host || n_tokens < 0) return BALANCEKV_E_INVAL;
+  if (n_tokens == 0) return BALANCEKV_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)c->cfg.n_seqs * c->cfg.n_kv_heads * n_tokens * c->cfg.head_dim * c->esz;
+  if (bytes > c->bounce_bytes) {
+    BKV_CUDA(cudaStreamSynchronize(st));
+    if (c->bounce_K) { cudaFree(c->bounce_K); cudaFree(c->bounce_V); c->bytes_resident -= 2 * c->bounce_bytes; }
+    c->bounce_K = c->bounce_V = nullptr; c->bounce_bytes = 0;
+    BKV_CUDA(cudaMalloc(&c->bounce_K, bytes));
+    BKV_CUDA(cudaMalloc(&c->bounce_V, bytes));
+    c->bounce_bytes = bytes; c->bytes_resident += 2 * bytes;
+  }
+  BKV_CUDA(cudaMemcpyAsync(c->bounce_K, K_host, bytes, cudaMemcpyHostToDevice, st));
+  BKV_CUDA(cudaMemcpyAsync(c->bounce_V, V_host, bytes, cudaMemcpyHostToDevice, st));
+  return append_impl(c, layer_streams(c, layer), 0, c->bounce_K, c->bounce_V, nullptr, n_tokens, st);
+}
+
+int balancekv_cache_load_level(balancekv_ctx* c, int layer, int level, const void* K, const void* V,
+                               const int32_t* orig_idx, int n_tokens, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
+  if (level != 0 && level != c->cfg.levels) return BALANCEKV_E_INVAL;
+  return append_impl(c, layer_streams(c, layer), level, K, V, orig_idx, n_tokens, static_cast<cudaStream_t>(stream));
+}
+
+// Runs one planned batch: per level radii -> walk -> selection/compaction, then the
+// level-0 remainder moves and the segment-table update.
+static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
+  const Geom& G = c->G;
+  for (int l = 0; l < G.T; ++l) {
+    std::vector<CallDesc>& calls = P.levels[l];
+    if (calls.empty()) continue;
+    if (c->debug)
+      for (CallDesc& d : calls) d.dbg_off = dbg_offset(c, d.stream, l, d.ordinal);
+    for (size_t first = 0; first < calls.size(); first += c->max_calls) {
+      const int n = (int)std::min<size_t>(c->max_calls, calls.size() - first);
+      void* d_calls = nullptr;
+      int rc = ring_push(c, calls.data() + first, (size_t)n * sizeof(CallDesc), st, &d_calls);
+      if (rc) return rc;
+      const CallDesc* dc = static_cast<const CallDesc*>(d_calls);
+      const bool need_radii = G.center_keys || G.fixed_rk2 <= 0.f || G.fixed_rv2 <= 0.f;
+      if (need_radii) {
+        BKV_CUDA(launch_radii(G, c->A, dc, n, c->d_stats, c->d_tokshift, st));
+        c->kernels_launched += 1 + (G.center_keys ? 1 : 0);
+      }
+      if (c->use_tc) {
+        BKV_CUDA(launch_walk_tc(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
+                                c->dbg_p, c->d_fail, c->d_status, c->tmaps, nullptr, st));
+      } else {
+        BKV_CUDA(launch_walk_simt(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
+                                  c->dbg_p, c->d_fail, st));
+      }
+      BKV_CUDA(launch_compact(G, c->A, dc, n, l, c->d_eta, st));
+      c->kernels_launched += 2;
+      c->calls_run += n;
+    }
+  }
+  if (!P.moves.empty()) {
+    void* d_moves = nullptr;
+    int rc = ring_push(c, P.moves.data(), P.moves.size() * sizeof(MoveDesc), st, &d_moves);
+    if (rc) return rc;
+    BKV_CUDA(launch_move(G, c->A, static_cast<const MoveDesc*>(d_moves), (int)P.moves.size(), P.max_move_rows, st));
+    c->kernels_launched++;
+  }
+  if (!P.segs.empty()) {
+    void* d_segs = nullptr;
+    int rc = ring_push(c, P.segs.data(), P.segs.size() * sizeof(SegUpdate), st, &d_segs);
+    if (rc) return rc;
+    BKV_CUDA(launch_seg_update(c->A, static_cast<const SegUpdate*>(d_segs), (int)P.segs.size(), st));
+    c->kernels_launched++;
+  }
+  return BALANCEKV_OK;
+}
+
+static int compress_streams(balancekv_ctx* c, const std::vector<int>& streams, int T, cudaStream_t st) {
+  if (T != c->cfg.levels) return BALANCEKV_E_INVAL;
+  for (int s : streams) c->st[s].pending = 0;
+  if (T == 0) return BALANCEKV_OK;
+  // greedy batches of at most max_calls level-0 calls
+  std::vector<int64_t> left(streams.size());
+  bool any = false;
+  for (size_t i = 0; i < streams.size(); ++i) { left[i] = ready_blocks(c->Lo, c->st[streams[i]]); any |= left[i] > 0; }
+  Plan P;
+  while (any) {
+    std::vector<std::pair<int, int>> runs;
+    int budget = c->max_calls;
+    any = false;
+    for (size_t i = 0; i < streams.size() && budget > 0; ++i) {
+      if (left[i] <= 0) continue;
+      const int take = (int)std::min<int64_t>(left[i], budget);
+      runs.emplace_back(streams[i], take);
+      left[i] -= take; budget -= take;
+    }
+    for (size_t i = 0; i < streams.size(); ++i) any |= left[i] > 0;
+    if (runs.empty()) break;
+    if (!plan_batch(c->Lo, c->st.data(), runs, P)) return BALANCEKV_E_STATE;
+    int rc = run_plan(c, P, st);
+    if (rc) return rc;
+  }
+  return BALANCEKV_OK;
+}
+
+int balancekv_compress(balancekv_ctx* c, int T, void* stream) {
+  if (!c) return BALANCEKV_E_INVAL;
+  std::vector<int> all(c->n_streams);
+  for (int i = 0; i < c->n_streams; ++i) all[i] = i;
+  return compress_streams(c, all, T, static_cast<cudaStream_t>(stream));
+}
+
+int balancekv_compress_layer(balancekv_ctx* c, int layer, int T, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
+  return compress_streams(c, layer_streams(c, layer), T, static_cast<cudaStream_t>(stream));
+}
+
+int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return BALANCEKV_E_INVAL;
+  if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
+  const balancekv_config& f = c->cfg;
+  int64_t max_rows = 0;
+  for (int s = 0; s < f.n_seqs; ++s)
+    for (int h = 0; h < f.n_kv_heads; ++h) {
+      const StreamState& S = c->st[stream_id(c, s, layer, h)];
+      int64_t rows = S.len0;
+      for (int l = 1; l <= f.levels; ++l) rows += S.lvl_len[l];
+      max_rows = std::max(max_rows, rows);
+    }
+  const int tile_tokens = 16384 / (f.head_dim * c->esz);
+  const int64_t tiles = (max_rows + tile_tokens - 1) / tile_tokens + f.levels;
+  const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
+  BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
+                         static_cast<cudaStream_t>(stream)));
+  c->kernels_launched++;
+  return BALANCEKV_OK;
+}
+
+int balancekv_decode_attn_host(balancekv_ctx* c, int layer, const void* q_host, void* out_host, void* stream) {
+  if (!c || !q_host || !out_host) return BALANCEKV_E_INVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)c->cfg.n_seqs * c->cfg.n_q_heads * c->cfg.head_dim * c->esz;
+  if (!c->bounce_q) {
+    BKV_CUDA(cudaMalloc(&c->bounce_q, bytes));
+    BKV_CUDA(cudaMalloc(&c->bounce_out, bytes));
+    c->bytes_resident += 2 * bytes;
+  }
+  BKV_CUDA(cudaMemcpyAsync(c->bounce_q, q_host, bytes, cudaMemcpyHostToDevice, st));
+  int rc = balancekv_decode_attn(c, layer, c->bounce_q, c->bounce_out, stream);
+  if (rc) return rc;
+  BKV_CUDA(cudaMemcpyAsync(out_host, c->bounce_out, bytes, cudaMemcpyDeviceToHost, st));
+  return BALANCEKV_OK;
+}
+
+int balancekv_level_sizes(balancekv_ctx* c, int seq, int layer, int kv_head, int32_t* sizes) {
+  if (!c || !sizes) return BALANCEKV_E_INVAL;
+  const balancekv_config& f = c->cfg;
+  if (seq < 0 || seq >= f.n_seqs || layer < 0 || layer >= f.n_layers || kv_head < 0 || kv_head >= f.n_kv_heads)
+    return BALANCEKV_E_INVAL;
+  const StreamState& S = c->st[stream_id(c, seq, layer, kv_head)];
+  sizes[0] = S.len0;
+  for (int l = 1; l <= f.levels; ++l) sizes[l] = S.lvl_len[l];
+  return BALANCEKV_OK;
+}
+
+int balancekv_cache_view(balancekv_ctx* c, int seq, int layer, int kv_head, const void** K, const void** V,
+                         const float** w, const int32_t** orig_idx, int* len) {
+  if (!c) return BALANCEKV_E_INVAL;
+  const balancekv_config& f = c->cfg;
+  if (seq < 0 || seq >= f.n_seqs || layer < 0 || layer >= f.n_layers || kv_head < 0 || kv_head >= f.n_kv_heads)
+    return BALANCEKV_E_INVAL;
+  BKV_CUDA(cudaDeviceSynchronize());
+  const int s = stream_id(c, seq, layer, kv_head);
+  const StreamState& S = c->st[s];
+  int64_t total = S.len0;
+  for (int l = 1; l <= f.levels; ++l) total += S.lvl_len[l];
+  if (total > c->view_cap) {
+    void* old[] = {c->view_K, c->view_V, c->view_w, c->view_idx};
+    for (void* p : old) if (p) cudaFree(p);
+    c->view_K = c->view_V = nullptr; c->view_w = nullptr; c->view_idx = nullptr;
+    const int64_t cap = std::max<int64_t>(total, 1024);
+    const size_t rb = (size_t)f.head_dim * c->esz;
+    BKV_CUDA(cudaMalloc(&c->view_K, cap * rb));
+    BKV_CUDA(cudaMalloc(&c->view_V, cap * rb));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->view_w), cap * sizeof(float)));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->view_idx), cap * sizeof(int32_t)));
+    c->view_cap = cap;
+  }
+  const size_t rb = (size_t)f.head_dim * c->esz;
+  int64_t pos = 0;
+  for (int l = f.levels; l >= 0; --l) {
+    const int64_t n = l == 0 ? S.len0 : S.lvl_len[l];
+    if (n == 0) continue;
+    const int64_t start = l == 0 ? S.start0 : (l == f.levels ? 0 : S.lvl_base[l]);
+    const int64_t row = (int64_t)s * c->Lo.R + c->Lo.region_off[l] + start;
+    BKV_CUDA(cudaMemcpy(static_cast<char*>(c->view_K) + pos * rb, static_cast<char*>(c->A.K) + row * rb, n * rb, cudaMemcpyDeviceToDevice));
+    BKV_CUDA(cudaMemcpy(static_cast<char*>(c->view_V) + pos * rb, static_cast<char*>(c->A.V) + row * rb, n * rb, cudaMemcpyDeviceToDevice));
+    BKV_CUDA(cudaMemcpy(c->view_idx + pos, c->A.idx + row, n * sizeof(int32_t), cudaMemcpyDeviceToDevice));
+    BKV_CUDA(launch_fill_weights(c->view_w + pos, (int)n, std::ldexp(1.0f, l), 0));
+    pos += n;
+  }
+  BKV_CUDA(cudaDeviceSynchronize());
+  if (K) *K = c->view_K;
+  if (V) *V = c->view_V;
+  if (w) *w = c->view_w;
+  if (orig_idx) *orig_idx = c->view_idx;
+  if (len) *len = (int)total;
+  return BALANCEKV_OK;
+}
+
+int balancekv_debug_enable(balancekv_ctx* c, int on) {
+  if (!c) return BALANCEKV_E_INVAL;
+  if (!on) { c->debug = false; return BALANCEKV_OK; }
+  if (c->cfg.levels == 0) return BALANCEKV_OK;
+  if (!c->dbg_eta) {
+    if (c->calls_run > 0) return BALANCEKV_E_STATE;
+    const int64_t blocks = c->cfg.max_tokens / c->cfg.block;
+    int64_t base = 0;
+    for (int l = 0; l < c->cfg.levels; ++l) { c->dbg_level_base[l] = base; base += blocks >> l; }
+    c->dbg_calls_per_stream = std::max<int64_t>(base, 1);
+    const size_t n = (size_t)c->n_streams * c->dbg_calls_per_stream * c->cfg.block;
+    int rc;
+    if ((rc = dev_alloc(c, &c->dbg_eta, n))) return rc;
+    if ((rc = dev_alloc(c, &c->dbg_S, n))) return rc;
+    if ((rc = dev_alloc(c, &c->dbg_p, n))) return rc;
+  }
+  c->debug = true;
+  return BALANCEKV_OK;
+}
+
+int balancekv_debug_call(balancekv_ctx* c, int seq, int layer, int kv_head, int level, int call_ordinal,
+                         const int8_t** eta, const float** S, const float** p, int* m) {
+  if (!c || !c->dbg_eta) return BALANCEKV_E_STATE;
+  const balancekv_config& f = c->cfg;
+  if (seq < 0 || seq >= f.n_seqs || layer < 0 || layer >= f.n_layers || kv_head < 0 || kv_head >= f.n_kv_heads)
+    return BALANCEKV_E_INVAL;
+  if (level < 0 || level >= f.levels) return BALANCEKV_E_INVAL;
+  const int s = stream_id(c, seq, layer, kv_head);
+  if (call_ordinal < 0 || call_ordinal >= c->st[s].calls_done[level]) return BALANCEKV_E_INVAL;
+  const int64_t off = dbg_offset(c, s, level, call_ordinal);
+  if (eta) *eta = c->dbg_eta + off;
+  if (S) *S = c->dbg_S + off;
+  if (p) *p = c->dbg_p + off;
+  if (m) *m = f.block;
+  return BALANCEKV_OK;
+}
+
+int balancekv_stats(balancekv_ctx* c, balancekv_stats_t* out) {
+  if (!c || !out) return BALANCEKV_E_INVAL;
+  BKV_CUDA(cudaDeviceSynchronize());
+  unsigned long long fails = 0;
+  int status = 0;
+  BKV_CUDA(cudaMemcpy(&fails, c->d_fail, sizeof(fails), cudaMemcpyDeviceToHost));
+  BKV_CUDA(cudaMemcpy(&status, c->d_status, sizeof(status), cudaMemcpyDeviceToHost));
+  int64_t stored = 0;
+  for (const StreamState& S : c->st) {
+    stored += S.len0;
+    for (int l = 1; l <= c->cfg.levels; ++l) stored += S.lvl_len[l];
+  }
+  out->tokens_appended = c->tokens_appended;
+  out->tokens_stored = stored;
+  out->calls_run = c->calls_run;
+  out->walk_fails = (int64_t)fails;
+  out->device_status = status;
+  out->bytes_resident = (int64_t)c->bytes_resident;
+  out->kernels_launched = c->kernels_launched;
+  return BALANCEKV_OK;
+}
+
+int balancekv_plan_calls(int block, int levels, int recent_window, const int32_t* appended_after_event, int n_events,
+                         int32_t* calls_out, int max_calls) {
+  if (block < 2 || block % 2 || levels < 0 || levels > kMaxLevels || recent_window < 0 || !appended_after_event ||
+      n_events < 0 || (!calls_out && max_calls > 0))
+    return BALANCEKV_E_INVAL;
+  Layout Lo;
+  Lo.t = block; Lo.T = levels; Lo.W = recent_window;
+  Lo.R = (int64_t)1 << 40;
+  for (int l = 0; l <= levels; ++l) Lo.region_off[l] = l * (1 << 20);
+  Lo.pool_row[0] = (int64_t)1 << 41; Lo.pool_row[1] = (int64_t)1 << 42;
+  Lo.pool_pairs = (int64_t)1 << 30;
+  StreamState S;
+  int n_out = 0;
+  Plan P;
+  for (int e = 0; e < n_events; ++e) {
+    if (appended_after_event[e] < S.appended) return BALANCEKV_E_INVAL;
+    S.len0 += (int32_t)(appended_after_event[e] - S.appended);
+    S.appended = appended_after_event[e];
+    if (levels == 0) continue;
+    const int64_t nb = ready_blocks(Lo, S);
+    if (nb <= 0) continue;
+    std::vector<std::pair<int, int>> runs{{0, (int)nb}};
+    if (!plan_batch(Lo, &S, runs, P)) return BALANCEKV_E_STATE;
+    // sequential order of Algorithm 3: block by block, climbing levels after each block
+    std::vector<size_t> next(levels, 0);
+    const int64_t first_block = S.calls_done[0] - nb;
+    for (int64_t b = 0; b < nb; ++b) {
+      int64_t beta = first_block + b + 1;
+      for (int l = 0; l < levels; ++l) {
+        if (next[l] >= P.levels[l].size()) break;
+        const CallDesc& d = P.levels[l][next[l]++];
+        if (n_out < max_calls) {
+          calls_out[3 * n_out] = e; calls_out[3 * n_out + 1] = l; calls_out[3 * n_out + 2] = d.ordinal;
+        }
+        ++n_out;
+        if (beta % 2) break;
+        beta /= 2;
+      }
+    }
+  }
+  return n_out;
+}
+
+}  // extern "C"

@@ -1,0 +1,186 @@
+// Data-movement and reduction helpers of the BalanceKV library:
+//   append / level load   (Algorithm 3: C^0 <- C^0 + {k_j, v_j})
+//   level-0 remainder move
+//   per-call radii r_key^2, r_value^2 (inputs of Algorithm 2) and the optional key shift
+#include "common.cuh"
+
+namespace bkv {
+
+namespace {
+
+constexpr int kCopyRows = 64;  // rows handled by one CTA of the copy kernels
+
+// Copies rows of 16-byte chunks: dst[r][c] = src[r][c].
+__device__ inline void copy_rows(uint4* __restrict__ dst, const uint4* __restrict__ src, int rows, int chunks) {
+  const int total = rows * chunks;
+  for (int i = threadIdx.x; i < total; i += blockDim.x) dst[i] = src[i];
+}
+
+__global__ void __launch_bounds__(256)
+append_kernel(Geom G, Arena A, const AppendDesc* __restrict__ descs, const void* __restrict__ Ksrc,
+              const void* __restrict__ Vsrc, const int32_t* __restrict__ idx_src) {
+  const AppendDesc D = descs[blockIdx.x];
+  const int row0 = blockIdx.y * kCopyRows;
+  if (row0 < D.n) {
+    const int rows = min(kCopyRows, D.n - row0);
+    const int esz = G.is_bf16 ? 2 : 4;
+    const int chunks = G.d * esz / 16;
+    const size_t dst_b = (size_t)(D.dst_row + row0) * G.d * esz;
+    const size_t src_b = ((size_t)D.src_off + (size_t)row0 * G.d) * esz;
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(Ksrc) + src_b), rows, chunks);
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(Vsrc) + src_b), rows, chunks);
+    for (int i = threadIdx.x; i < rows; i += blockDim.x)
+      A.idx[D.dst_row + row0 + i] = idx_src ? idx_src[D.src_off / G.d + row0 + i] : D.idx0 + row0 + i;
+  }
+  if (blockIdx.y == 0 && threadIdx.x == 0) A.seg[(size_t)D.stream * (G.T + 1) + D.level].len = D.new_len;
+}
+
+__global__ void __launch_bounds__(256)
+move_kernel(Geom G, Arena A, const MoveDesc* __restrict__ descs) {
+  const MoveDesc D = descs[blockIdx.x];
+  const int row0 = blockIdx.y * kCopyRows;
+  if (row0 < D.n) {
+    const int rows = min(kCopyRows, D.n - row0);
+    const int esz = G.is_bf16 ? 2 : 4;
+    const int chunks = G.d * esz / 16;
+    const size_t dst_b = (size_t)(D.dst_row + row0) * G.d * esz;
+    const size_t src_b = (size_t)(D.src_row + row0) * G.d * esz;
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(A.K) + src_b), rows, chunks);
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(A.V) + src_b), rows, chunks);
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) A.idx[D.dst_row + row0 + i] = A.idx[D.src_row + row0 + i];
+  }
+}
+
+__global__ void seg_update_kernel(Arena A, const SegUpdate* __restrict__ ups, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) A.seg[ups[i].index] = Seg{ups[i].start, ups[i].len};
+}
+
+// Column means of the call's keys, one CTA per call, thread e owns column e
+// (fixed summation order, so the result is reproducible).
+template <bool kBf16>
+__global__ void mean_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, float* __restrict__ mean) {
+  const CallDesc C = calls[blockIdx.x];
+  const int e = threadIdx.x;
+  if (e >= G.d) return;
+  float s = 0.f;
+  for (int j = 0; j < G.t; ++j) {
+    const size_t off = (size_t)(C.src_row + j) * G.d + e;
+    s += kBf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(A.K)[off]) : static_cast<const float*>(A.K)[off];
+  }
+  mean[(size_t)blockIdx.x * G.d + e] = s / (float)G.t;
+}
+
+// r_key^2 = max_j ||k_j - mean||^2, r_value^2 = max_j ||v_j||^2 over the call's tokens,
+// and the per-token shift a_j = <k_j, mean> - ||mean||^2/2, with which
+// <k_i - mean, k_j - mean> = <k_i, k_j> - a_i - a_j.
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+radii_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, CallStat* __restrict__ stats,
+             const float* __restrict__ mean, float* __restrict__ tok_shift) {
+  const CallDesc C = calls[blockIdx.x];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int esz = kBf16 ? 2 : 4;
+  float mk = 0.f, mv = 0.f;
+  const float* mu = mean ? mean + (size_t)blockIdx.x * G.d : nullptr;
+  float mu2 = 0.f;
+  if (mu) {
+    for (int e = lane; e < G.d; e += 32) mu2 += mu[e] * mu[e];
+    mu2 = warp_sum(mu2);
+  }
+  for (int r = blockIdx.y * 64 + warp; r < min(G.t, (int)(blockIdx.y + 1) * 64); r += 8) {
+    const char* krow = static_cast<const char*>(A.K) + (size_t)(C.src_row + r) * G.d * esz;
+    const char* vrow = static_cast<const char*>(A.V) + (size_t)(C.src_row + r) * G.d * esz;
+    float sk = 0.f, sv = 0.f, sm = 0.f;
+    for (int e = lane * 8; e < G.d; e += 256) {
+      float a[8], b[8];
+      load8<kBf16>(krow, e, a);
+      load8<kBf16>(vrow, e, b);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        sk = fmaf(a[i], a[i], sk);
+        sv = fmaf(b[i], b[i], sv);
+        if (mu) sm = fmaf(a[i], mu[e + i], sm);
+      }
+    }
+    sk = warp_sum(sk); sv = warp_sum(sv);
+    if (mu) {
+      sm = warp_sum(sm);
+      const float shift = sm - 0.5f * mu2;
+      sk = fmaxf(sk - 2.f * shift, 0.f);
+      if (lane == 0) tok_shift[(size_t)blockIdx.x * G.t + r] = shift;
+    }
+    mk = fmaxf(mk, sk); mv = fmaxf(mv, sv);
+  }
+  __shared__ float smk[8], smv[8];
+  if (lane == 0) { smk[warp] = mk; smv[warp] = mv; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) { mk = fmaxf(mk, smk[w]); mv = fmaxf(mv, smv[w]); }
+    // non-negative floats order like their bit patterns
+    atomicMax(reinterpret_cast<int*>(&stats[blockIdx.x].rk2), __float_as_int(mk));
+    atomicMax(reinterpret_cast<int*>(&stats[blockIdx.x].rv2), __float_as_int(mv));
+  }
+}
+
+__global__ void fill_weights_kernel(float* w, int n, float value) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) w[i] = value;
+}
+
+}  // namespace
+
+cudaError_t launch_append(const Geom& G, const Arena& A, const AppendDesc* descs, int n_desc, int max_rows,
+                          const void* Ksrc, const void* Vsrc, const int32_t* idx_src, cudaStream_t st) {
+  if (n_desc <= 0) return cudaSuccess;
+  dim3 grid(n_desc, (max_rows + kCopyRows - 1) / kCopyRows);
+  if (grid.y == 0) grid.y = 1;
+  append_kernel<<<grid, 256, 0, st>>>(G, A, descs, Ksrc, Vsrc, idx_src);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_move(const Geom& G, const Arena& A, const MoveDesc* descs, int n_desc, int max_rows,
+                        cudaStream_t st) {
+  if (n_desc <= 0) return cudaSuccess;
+  dim3 grid(n_desc, (max_rows + kCopyRows - 1) / kCopyRows);
+  if (grid.y == 0) grid.y = 1;
+  move_kernel<<<grid, 256, 0, st>>>(G, A, descs);
+  return cudaGetLastError();
+}
+
+// stats must hold n_calls entries; tok_shift n_calls * t floats (+ n_calls * d floats of
+// mean scratch behind it) when key centering is on, else it may be null.
+cudaError_t launch_radii(const Geom& G, const Arena& A, const CallDesc* calls, int n_calls, CallStat* stats,
+                         float* tok_shift, cudaStream_t st) {
+  if (n_calls <= 0) return cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(stats, 0, sizeof(CallStat) * (size_t)n_calls, st);
+  if (e != cudaSuccess) return e;
+  float* mean = nullptr;
+  if (G.center_keys) {
+    mean = tok_shift + (size_t)n_calls * G.t;
+    if (G.is_bf16) mean_kernel<true><<<n_calls, 128, 0, st>>>(G, A, calls, mean);
+    else mean_kernel<false><<<n_calls, 128, 0, st>>>(G, A, calls, mean);
+  }
+  dim3 grid(n_calls, (G.t + 63) / 64);
+  if (G.is_bf16) radii_kernel<true><<<grid, 256, 0, st>>>(G, A, calls, stats, mean, tok_shift);
+  else radii_kernel<false><<<grid, 256, 0, st>>>(G, A, calls, stats, mean, tok_shift);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_seg_update(const Arena& A, const SegUpdate* ups, int n, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  seg_update_kernel<<<(n + 255) / 256, 256, 0, st>>>(A, ups, n);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill_weights(float* w, int n, float value, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  fill_weights_kernel<<<(n + 255) / 256, 256, 0, st>>>(w, n, value);
+  return cudaGetLastError();
+}
+
+}  // namespace bkv
