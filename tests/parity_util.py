@@ -116,6 +116,7 @@ class Harness:
     def check_all(self, s_tol_rel, streams=None, s_tol_abs=1e-6):
         tot = marg = 0
         self.oracles = {}
+        self.recs = {}
         for seq in range(self.B):
             for layer in range(self.L):
                 for head in range(self.H):
@@ -129,6 +130,7 @@ class Harness:
                     tot += n
                     marg += m
                     self.oracles[(seq, layer, head)] = forced
+                    self.recs[(seq, layer, head)] = rec
         assert marg <= 1e-3 * max(tot, 1), (marg, tot)
         return tot, marg
 

@@ -89,13 +89,12 @@ def test_student_t_keys_window_and_three_levels_streamed_in_chunks(cuda_lib):
         q = synth.queries(1004, 0, step, B, H * g, d, "bf16")
         hz.check_decode(0, q, DEC_TOL["bf16"])
         hz.append_layer(0, K[:, 0, :, n + step:n + step + 1], V[:, 0, :, n + step:n + step + 1])   # decode-phase token
-        for o in hz.oracles.values():
-            pass
-        hz.oracles = {k: hz.oracle_replay(*k, rec=None) for k in hz.oracles}   # no new calls: replay is cheap
-        # replay without forcing is only valid if the GPU's signs equal the oracle's own; check that
+        # no new calls fire (compress is not called in the decode phase): replay with the same signs
+        hz.oracles = {k: hz.oracle_replay(*k, rec=hz.recs[k]) for k in hz.oracles}
         for (s_, l_, h_), o in hz.oracles.items():
             Kg, Vg, wg, ig = hz.ctx.cache_view(s_, l_, h_)
             assert np.array_equal(ig.cpu().numpy(), o.view()[3])
+            assert np.all(wg.cpu().numpy()[-(step + 1):] == 1.0)
 
 
 def test_T0_is_exact_attention_and_empty_streams_give_zeros(cuda_lib):
