@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the BalanceKV hot path on B200.
+
+One *step* = one pass of the whole hot path over one batch of synthetic input shaped like one
+Llama-3.1-8B layer: append the 32768-token context of 8 KV heads (bf16, d=128), compress it
+with blocks of 1024 and T=2, then 256 decode steps, each appending one uncompressed token per
+stream and running decode attention for the 32 query heads over the weighted cache.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+prints one JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD = dict(name="llama3.1-8b-layer", n_seqs=1, n_layers=1, n_kv_heads=8, n_q_heads=32, head_dim=128, dtype="bf16",
+                context=32768, block=1024, levels=2, decode_steps=256, recipe="llama", data_seed=1002, walk_seed=0)
+METRIC = "compressed_kv_tokens_per_s"
+UNIT = "KV token-heads/s through append+compress(T=2)+256 decode steps"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=float(j["hbm_gbs"]), tensor=float(j["bf16_tflops"]), tensor_sustained=float(j["bf16_tflops_sustained"]),
+                    source="measured")
+    return dict(hbm=6650.0, tensor=1590.0, tensor_sustained=1400.0, source="fallback")
+
+
+def make_inputs(w, n_context, n_decode):
+    """Host tensors (float32 values already rounded to bf16): context K,V, decode K,V, queries."""
+    from paper_2502_07861_b200 import synth
+
+    B, H, d = w["n_seqs"], w["n_kv_heads"], w["head_dim"]
+    K = np.empty((B, H, n_context + n_decode, d), np.float32)
+    V = np.empty_like(K)
+    for b in range(B):
+        for h in range(H):
+            K[b, h], V[b, h] = synth.stream_kv(w["recipe"], w["data_seed"], b, 0, h, n_context + n_decode, d, w["dtype"])
+    q = np.stack([synth.queries(w["data_seed"], 0, s, B, w["n_q_heads"], d, w["dtype"]) for s in range(n_decode)])
+    return K, V, q
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample(w, K, V, q, sample_tokens, decode_steps):
+    """The oracle, as it stands, on the first `sample_tokens` tokens of every stream plus
+    `decode_steps` decode steps; returns (seconds, token-heads, threads)."""
+    import oracle
+
+    B, H, d, g = w["n_seqs"], w["n_kv_heads"], w["head_dim"], w["n_q_heads"] // w["n_kv_heads"]
+    t0 = time.perf_counter()
+    streams = []
+    for b in range(B):
+        for h in range(H):
+            o = oracle.OracleStream(oracle.OracleParams(d=d, t=w["block"], T=w["levels"], layer=0, head=h,
+                                                        max_tokens=w["context"] + w["decode_steps"], seed=w["walk_seed"] + b))
+            o.append(K[b, h, :sample_tokens], V[b, h, :sample_tokens])
+            streams.append((b, h, o))
+    oracle.compress_streams([s[2] for s in streams])
+    n_ctx = w["context"]
+    for s in range(decode_steps):
+        for b, h, o in streams:
+            o.append(K[b, h, n_ctx + s:n_ctx + s + 1], V[b, h, n_ctx + s:n_ctx + s + 1])
+            o.decode(q[s, b, h * g:(h + 1) * g])
+    dt = time.perf_counter() - t0
+    return dt, B * H * sample_tokens, oracle.num_threads()
+
+
+def run_reference(args, w):
+    """CPU oracle arm: each step is a bounded sample (1/8 of the context per stream)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample, dsteps = w["context"] // 8, w["decode_steps"] // 8
+    K, V, q = make_inputs(w, w["context"], w["decode_steps"])
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, K, V, q, w["block"] * 2, 1)
+    times = []
+    for _ in range(args.steps):
+        dt, units, threads = oracle_sample(w, K, V, q, sample, dsteps)
+        times.append(dt)
+    val = units * len(times) / sum(times)
+    sample_txt = f"first {sample} of {w['context']} context tokens of each of the {w['n_kv_heads']} streams + {dsteps} decode steps"
+    line = dict(metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * float(np.mean(times)), higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=w["name"], sample=sample_txt, context=w["context"], block=w["block"], levels=w["levels"]),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=threads, kind="oracle", sample=sample_txt),
+                e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="balancekv")
+    ap.add_argument("--gram-path", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--context", type=int, default=None, help="override the context length (profiling a small case)")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    args = ap.parse_args()
+    w = dict(WORKLOAD)
+    if args.context:
+        w["context"] = args.context
+    if args.decode_steps is not None:
+        w["decode_steps"] = args.decode_steps
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2502_07861_b200 as bk
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    args.warmup = max(args.warmup, 3)
+
+    # every rank owns an independent replica of the workload (streams shard with no exchange)
+    w["data_seed"] = WORKLOAD["data_seed"] + 100 * rank
+    B, H, Hq, d = w["n_seqs"], w["n_kv_heads"], w["n_q_heads"], w["head_dim"]
+    n_ctx, n_dec, T, t = w["context"], w["decode_steps"], w["levels"], w["block"]
+    Kf, Vf, qf = make_inputs(w, n_ctx, n_dec)
+    bf = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16)
+    K_ctx_h = bf(Kf[:, :, :n_ctx]).pin_memory()
+    V_ctx_h = bf(Vf[:, :, :n_ctx]).pin_memory()
+    K_dec_h = bf(np.moveaxis(Kf[:, :, n_ctx:], 2, 0)[:, :, :, None, :]).pin_memory()   # [steps, B, H, 1, d]
+    V_dec_h = bf(np.moveaxis(Vf[:, :, n_ctx:], 2, 0)[:, :, :, None, :]).pin_memory()
+    q_h = bf(qf).pin_memory()                                                          # [steps, B, Hq, d]
+    out_h = torch.empty_like(q_h).pin_memory()
+    K_ctx, V_ctx, K_dec, V_dec, q_d = (x.cuda() for x in (K_ctx_h, V_ctx_h, K_dec_h, V_dec_h, q_h))
+    out_d = torch.empty(B, Hq, d, dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    ctx = bk.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, head_dim=d, dtype="bf16", block=t, levels=T,
+                     max_tokens=n_ctx + n_dec, seed=w["walk_seed"] + rank, gram_path=args.gram_path)
+
+    def step_device(ev=None):
+        ctx.reset()
+        if ev: ev[0].record()
+        ctx.stream_append_layer(0, K_ctx, V_ctx)
+        ctx.compress()
+        if ev: ev[1].record()
+        for s in range(n_dec):
+            ctx.stream_append_layer(0, K_dec[s], V_dec[s])
+            ctx.decode_attn(0, q_d[s], out_d)
+        if ev: ev[2].record()
+
+    def step_host():
+        ctx.reset()
+        ctx.stream_append_layer_host(0, K_ctx_h, V_ctx_h)
+        ctx.compress()
+        for s in range(n_dec):
+            ctx.stream_append_layer_host(0, K_dec_h[s], V_dec_h[s])
+            ctx.decode_attn_host(0, q_h[s], out_h[s])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.fill_(1)
+        step_device()
+    launches_before = ctx.stats()["kernels_launched"]
+    ctx.profile_enable(True)
+    ctx.profile_read()
+    sampler = ClockSampler(local)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    sampler.start()
+    for i in range(args.steps):
+        flush.fill_(i & 255)       # L2 flush between timed iterations (outside the event brackets)
+        step_device(evs[i])
+    barrier()
+    clocks = sampler.stop()
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    launches = ctx.stats()["kernels_launched"] - launches_before
+    t_step = np.array([e[0].elapsed_time(e[2]) for e in evs])           # ms
+    t_comp = np.array([e[0].elapsed_time(e[1]) for e in evs])
+    t_dec = np.array([e[1].elapsed_time(e[2]) for e in evs])
+    total_ms = float(t_step.sum())
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    units_per_step = B * H * n_ctx
+    value = world * units_per_step * args.steps / (total_ms * 1e-3)
+
+    # end to end through the host-buffer entry points (pinned host memory in, host out)
+    for _ in range(2):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps = max(2, min(args.steps, 5))
+    for i in range(e2e_steps):
+        step_host()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_s = float(tt.item())
+    esz = 2
+    h2d = 2 * B * H * (n_ctx + n_dec) * d * esz + n_dec * B * Hq * d * esz
+    d2h = n_dec * B * Hq * d * esz
+    status = ctx.stats()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    calls0, calls1 = n_ctx // t, (n_ctx // t) // 2
+    n_calls = B * H * sum((n_ctx // t) >> l for l in range(T))
+    # algorithmic work: strict lower triangle of two Gram matrices per call
+    flop_per_call = 2.0 * (t * (t - 1) / 2.0) * 2.0 * d
+    gw_n, gw_ms = prof["gram_walk"]
+    gw_ms_per_launch = gw_ms / max(gw_n, 1)
+    calls_per_launch = n_calls * args.steps / max(gw_n, 1)
+    tensor_ach = flop_per_call * calls_per_launch / (gw_ms_per_launch * 1e-3) / 1e12 if gw_n else 0.0
+    # compaction: per call read t/2 rows of K and V, write t/2 rows, t sign bytes, 2 index words per survivor
+    cp_n, cp_ms = prof["compact"]
+    cp_bytes = (t // 2) * (2 * 2 * d * esz + 8) + t
+    cp_gbs = cp_bytes * n_calls * args.steps / (cp_ms * 1e-3) / 1e9 if cp_n else 0.0
+    # decode: every stored row of K and V once per launch
+    dc_n, dc_ms = prof["decode"]
+    stored0 = n_ctx >> T
+    dec_bytes_total = sum(B * H * (stored0 + s + 1) * 2 * d * esz for s in range(n_dec)) * args.steps
+    dc_gbs = dec_bytes_total / (dc_ms * 1e-3) / 1e9 if dc_n else 0.0
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        sample, dsteps = n_ctx // 8, max(n_dec // 8, 1) if n_dec else 0
+        dt, units, threads = oracle_sample(w, Kf, Vf, qf, sample, dsteps)
+        cpu = dict(value=units / dt, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
+                   sample=f"first {sample} of {n_ctx} context tokens of each of the {B * H} streams + {dsteps} decode steps")
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+        data="synthetic",
+        config=dict(workload=w["name"], n_kv_heads=H, n_q_heads=Hq, head_dim=d, context=n_ctx, block=t, levels=T,
+                    decode_steps=n_dec, gram_path="tcgen05" if False else ("auto" if args.gram_path == 0 else args.gram_path),
+                    l2="flushed between steps (256 MB write, outside the event brackets); inputs 134 MB > L2",
+                    replicas_per_gpu=1),
+        compress_tokens_per_s=units_per_step / (float(t_comp.mean()) * 1e-3),
+        compress_ms=float(t_comp.mean()),
+        decode_us_per_step=1e3 * float(t_dec.mean()) / max(n_dec, 1),
+        decode_attn_kernel_us=1e3 * dc_ms / max(dc_n, 1),
+        roofline=dict(kernel="gram_walk", bound="tensor", achieved=tensor_ach, peak=peaks["tensor"], unit="TFLOP/s",
+                      frac=tensor_ach / peaks["tensor"], traffic=None, peak_source=peaks["source"],
+                      ms_per_launch=gw_ms_per_launch, launches=gw_n),
+        kernels=dict(
+            compact=dict(bound="hbm", achieved=cp_gbs, peak=peaks["hbm"], unit="GB/s", frac=cp_gbs / peaks["hbm"],
+                         ms_per_launch=cp_ms / max(cp_n, 1), launches=cp_n),
+            decode=dict(bound="hbm", achieved=dc_gbs, peak=peaks["hbm"], unit="GB/s", frac=dc_gbs / peaks["hbm"],
+                        us_per_launch=1e3 * dc_ms / max(dc_n, 1), launches=dc_n),
+            radii_ms=prof["radii"][1] / args.steps, append_ms=prof["append"][1] / args.steps,
+            bookkeeping_ms=prof["bookkeeping"][1] / args.steps),
+        e2e=dict(value=world * units_per_step * e2e_steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                 ms_per_step=1e3 * e2e_s / e2e_steps, timing="wall clock, synchronised on both sides"),
+        gpu_launches=int(launches), clocks=clocks, cpu_baseline=cpu,
+        device_status=int(status["device_status"]), walk_fails=int(status["walk_fails"]),
+    )
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

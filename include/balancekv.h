@@ -144,6 +144,21 @@ int balancekv_debug_call(balancekv_ctx* ctx, int seq, int layer, int kv_head, in
                          int call_ordinal, const int8_t** eta, const float** S, const float** p,
                          int* m);
 
+/* Forget every token of every stream (Algorithm 3's "initialize C^i to empty"); memory,
+ * configuration and debug buffers are kept.  Enqueued on `stream`. */
+int balancekv_reset(balancekv_ctx* ctx, void* stream);
+
+/* Kernel timing for roofline reports.  While enabled, every launch of the kernel classes
+ * below is bracketed by CUDA events on its launch stream (at most 8192 launches between two
+ * reads; later ones are not recorded).  balancekv_profile_read synchronises the device and
+ * writes, per class, {launches, total milliseconds} into out_host[2*class + {0,1}], then
+ * clears the record.  Classes: 0 append/load, 1 radii (inputs of Algorithm 2), 2 Gram tiles +
+ * sign walk (Algorithm 2), 3 strict-half selection + compaction, 4 decode attention
+ * (Algorithm 1's output ratio), 5 bookkeeping (remainder move, segment table). */
+#define BALANCEKV_PROFILE_CLASSES 6
+int balancekv_profile_enable(balancekv_ctx* ctx, int on);
+int balancekv_profile_read(balancekv_ctx* ctx, double* out_host);
+
 int balancekv_stats(balancekv_ctx* ctx, balancekv_stats_t* out);
 const char* balancekv_strerror(int code);
 

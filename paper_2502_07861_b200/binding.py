@@ -20,8 +20,10 @@ EXPORTS = [
     "balancekv_stream_append_layer_host", "balancekv_compress", "balancekv_compress_layer",
     "balancekv_decode_attn", "balancekv_decode_attn_host", "balancekv_cache_load_level",
     "balancekv_cache_view", "balancekv_level_sizes", "balancekv_debug_enable", "balancekv_debug_call",
-    "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls",
+    "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
+    "balancekv_profile_enable", "balancekv_profile_read",
 ]
+PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
 
 class BalanceKVError(RuntimeError):
@@ -78,6 +80,9 @@ def load():
     lib.balancekv_strerror.argtypes = [ci]
     lib.balancekv_strerror.restype = C.c_char_p
     lib.balancekv_plan_calls.argtypes = [ci, ci, ci, vp, ci, vp, ci]
+    lib.balancekv_reset.argtypes = [vp, vp]
+    lib.balancekv_profile_enable.argtypes = [vp, ci]
+    lib.balancekv_profile_read.argtypes = [vp, vp]
     for name in EXPORTS:
         if name != "balancekv_strerror":
             getattr(lib, name).restype = ci
@@ -248,6 +253,18 @@ class Context:
         torch.cuda.synchronize()
         return (_from_ptr(pe.value, (m.value,), torch.int8), _from_ptr(ps.value, (m.value,), torch.float32),
                 _from_ptr(pp.value, (m.value,), torch.float32))
+
+    def reset(self, stream=None):
+        _check(self.lib.balancekv_reset(self._h, _stream_ptr(stream)), "balancekv_reset")
+
+    def profile_enable(self, on=True):
+        _check(self.lib.balancekv_profile_enable(self._h, 1 if on else 0), "balancekv_profile_enable")
+
+    def profile_read(self):
+        """{class name: (launches, total ms)} since the last read."""
+        buf = (C.c_double * (2 * len(PROFILE_CLASSES)))()
+        _check(self.lib.balancekv_profile_read(self._h, buf), "balancekv_profile_read")
+        return {n: (int(buf[2 * i]), float(buf[2 * i + 1])) for i, n in enumerate(PROFILE_CLASSES)}
 
     def stats(self):
         s = Stats()

@@ -83,7 +83,31 @@ struct balancekv_ctx {
   void* bounce_out = nullptr;
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
+
+  // optional per-class kernel timing
+  bool profiling = false;
+  std::vector<cudaEvent_t> prof_ev;     // pairs
+  std::vector<int> prof_class;
+  size_t prof_used = 0;
 };
+
+namespace {
+constexpr size_t kProfMax = 8192;
+// Brackets one kernel-class launch with events while profiling is on.
+struct ProfScope {
+  balancekv_ctx* c; cudaStream_t st; bool on;
+  ProfScope(balancekv_ctx* c_, int cls, cudaStream_t st_) : c(c_), st(st_), on(false) {
+    if (c->profiling && c->prof_used < kProfMax) {
+      on = true;
+      c->prof_class[c->prof_used] = cls;
+      cudaEventRecord(c->prof_ev[2 * c->prof_used], st);
+    }
+  }
+  ~ProfScope() {
+    if (on) { cudaEventRecord(c->prof_ev[2 * c->prof_used + 1], st); c->prof_used++; }
+  }
+};
+}  // namespace
 
 namespace {
 
@@ -285,6 +309,7 @@ int balancekv_destroy(balancekv_ctx* c) {
   if (c->h_ring) cudaFreeHost(c->h_ring);
   for (int i = 0; i < 2; ++i)
     if (c->ring_ev[i]) cudaEventDestroy(c->ring_ev[i]);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return BALANCEKV_OK;
 }
@@ -333,7 +358,10 @@ static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int le
   void* d_descs = nullptr;
   int rc = ring_push(c, descs.data(), descs.size() * sizeof(AppendDesc), st, &d_descs);
   if (rc) return rc;
-  BKV_CUDA(launch_append(c->G, c->A, static_cast<const AppendDesc*>(d_descs), (int)descs.size(), n, K, V, idx, st));
+  {
+    ProfScope ps(c, 0, st);
+    BKV_CUDA(launch_append(c->G, c->A, static_cast<const AppendDesc*>(d_descs), (int)descs.size(), n, K, V, idx, st));
+  }
   c->kernels_launched++;
   return BALANCEKV_OK;
 }
@@ -403,17 +431,23 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
       const CallDesc* dc = static_cast<const CallDesc*>(d_calls);
       const bool need_radii = G.center_keys || G.fixed_rk2 <= 0.f || G.fixed_rv2 <= 0.f;
       if (need_radii) {
+        ProfScope ps(c, 1, st);
         BKV_CUDA(launch_radii(G, c->A, dc, n, c->d_stats, c->d_tokshift, st));
         c->kernels_launched += 1 + (G.center_keys ? 1 : 0);
       }
       if (c->use_tc) {
+        ProfScope ps(c, 2, st);
         BKV_CUDA(launch_walk_tc(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
                                 c->dbg_p, c->d_fail, c->d_status, c->tmaps, nullptr, st));
       } else {
+        ProfScope ps(c, 2, st);
         BKV_CUDA(launch_walk_simt(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
                                   c->dbg_p, c->d_fail, st));
       }
-      BKV_CUDA(launch_compact(G, c->A, dc, n, l, c->d_eta, st));
+      {
+        ProfScope ps(c, 3, st);
+        BKV_CUDA(launch_compact(G, c->A, dc, n, l, c->d_eta, st));
+      }
       c->kernels_launched += 2;
       c->calls_run += n;
     }
@@ -422,6 +456,7 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
     void* d_moves = nullptr;
     int rc = ring_push(c, P.moves.data(), P.moves.size() * sizeof(MoveDesc), st, &d_moves);
     if (rc) return rc;
+    ProfScope ps(c, 5, st);
     BKV_CUDA(launch_move(G, c->A, static_cast<const MoveDesc*>(d_moves), (int)P.moves.size(), P.max_move_rows, st));
     c->kernels_launched++;
   }
@@ -429,6 +464,7 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
     void* d_segs = nullptr;
     int rc = ring_push(c, P.segs.data(), P.segs.size() * sizeof(SegUpdate), st, &d_segs);
     if (rc) return rc;
+    ProfScope ps(c, 5, st);
     BKV_CUDA(launch_seg_update(c->A, static_cast<const SegUpdate*>(d_segs), (int)P.segs.size(), st));
     c->kernels_launched++;
   }
@@ -490,8 +526,11 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
   const int tile_tokens = 16384 / (f.head_dim * c->esz);
   const int64_t tiles = (max_rows + tile_tokens - 1) / tile_tokens + f.levels;
   const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
-  BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
-                         static_cast<cudaStream_t>(stream)));
+  {
+    ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
+    BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
+                           static_cast<cudaStream_t>(stream)));
+  }
   c->kernels_launched++;
   return BALANCEKV_OK;
 }
@@ -602,6 +641,39 @@ int balancekv_debug_call(balancekv_ctx* c, int seq, int layer, int kv_head, int 
   if (S) *S = c->dbg_S + off;
   if (p) *p = c->dbg_p + off;
   if (m) *m = f.block;
+  return BALANCEKV_OK;
+}
+
+int balancekv_reset(balancekv_ctx* c, void* stream) {
+  if (!c) return BALANCEKV_E_INVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (StreamState& S : c->st) S = StreamState();
+  BKV_CUDA(cudaMemsetAsync(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (c->cfg.levels + 1), st));
+  return BALANCEKV_OK;
+}
+
+int balancekv_profile_enable(balancekv_ctx* c, int on) {
+  if (!c) return BALANCEKV_E_INVAL;
+  if (on && c->prof_ev.empty()) {
+    c->prof_ev.resize(2 * kProfMax);
+    c->prof_class.resize(kProfMax);
+    for (cudaEvent_t& e : c->prof_ev) BKV_CUDA(cudaEventCreate(&e));
+  }
+  c->profiling = on != 0;
+  return BALANCEKV_OK;
+}
+
+int balancekv_profile_read(balancekv_ctx* c, double* out) {
+  if (!c || !out) return BALANCEKV_E_INVAL;
+  BKV_CUDA(cudaDeviceSynchronize());
+  for (int i = 0; i < 2 * BALANCEKV_PROFILE_CLASSES; ++i) out[i] = 0.0;
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    float ms = 0.f;
+    BKV_CUDA(cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]));
+    out[2 * c->prof_class[i]] += 1.0;
+    out[2 * c->prof_class[i] + 1] += ms;
+  }
+  c->prof_used = 0;
   return BALANCEKV_OK;
 }
 
