@@ -1,22 +1,469 @@
-// SoftmaxBalance (Algorithm 2) with the Gram tiles on the tensor cores (tcgen05 / TMEM / TMA).
+// SoftmaxBalance (Algorithm 2) with the Gram tiles on the 5th-generation tensor cores.
+//
+// One CTA per call.  The call's t x t kernel matrix
+//   Ghat_ij = exp((<k_i,k_j> - r_key^2)/sqrt d) <v_i,v_j> / r_value^2      (proof of Theorem 3.2)
+// is visited in 128 x 128 tiles of its lower triangle, row panel by row panel.  For a tile,
+// TMA brings the bf16 rows of K and V into 128B-swizzled shared memory, one thread issues
+// tcgen05.mma (bf16 x bf16 -> fp32) for K_r K_c^T and V_r V_c^T into two TMEM accumulators,
+// and an epilogue warpgroup (thread = row) reads them back with tcgen05.ld, applies
+// exp2/scale/product and folds the tile into the row's running correlation
+//   S_j = sum_{i<j} eta_i Ghat_ij
+// with the signs of earlier panels.  The diagonal tile feeds the sequential walk: warp q owns
+// rows 32q..32q+31 of the panel, lane l owns one token, signs travel by warp shuffle,
+//   eta_j = +1  iff  u_j < 1/2 - S_j/(2c)  <=>  S_j < c (1 - 2 u_j),
+// u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).
+// TMEM is double buffered (2 x 256 columns), so the tensor core works on the next tile while
+// the epilogue drains the previous one; Ghat never touches global memory.
+//
+// Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
+// roles leave their loops, TMEM is freed and the kernel returns.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace bkv {
 
-bool walk_tc_supported(const Geom& G) { (void)G; return false; }
+namespace {
 
-cudaError_t walk_tc_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** tmaps_out) {
-  (void)G; (void)A; (void)total_rows;
-  *tmaps_out = nullptr;
-  return cudaErrorNotSupported;
+constexpr int kTile = 128;
+constexpr int kThreads = 192;              // warps 0-3: epilogue + walk, warp 4: TMA, warp 5: MMA
+constexpr uint32_t kHalfBytes = 16384;     // [128 rows][64 bf16] = one swizzle-atom column of a tile
+constexpr uint32_t kTileBytes = 32768;     // [128 rows][128 bf16]
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitCycles = 4000000000LL;
+
+struct TensorMaps {
+  CUtensorMap k, v;
+};
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ inline void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ inline void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ inline int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+__device__ inline void st_release(int* p, int v) {
+  asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+// Bounded wait on an mbarrier phase; false = gave up (abort flag set) or someone else aborted.
+__device__ inline bool wait_bar(uint64_t* bar, uint32_t parity, int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (ld_acquire(abort_flag)) return false;
+    if (clock64() - t0 > kWaitCycles) { st_release(abort_flag, 1); return false; }
+  }
+  return true;
+}
+// Bounded wait until *progress >= need.
+__device__ inline bool wait_progress(const int* progress, int need, int* abort_flag) {
+  if (ld_acquire(progress) >= need) return true;
+  const long long t0 = clock64();
+  while (ld_acquire(progress) < need) {
+    if (ld_acquire(abort_flag)) return false;
+    if (clock64() - t0 > kWaitCycles) { st_release(abort_flag, 1); return false; }
+  }
+  return true;
 }
 
-void walk_tc_release(void* tmaps) { (void)tmaps; }
+__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
 
-cudaError_t launch_walk_tc(const Geom&, const Arena&, const CallDesc*, int, int, const CallStat*, const float*,
-                           int8_t*, int8_t*, float*, float*, unsigned long long*, int*, const void*, const void*,
-                           cudaStream_t) {
-  return cudaErrorNotSupported;
+// Shared-memory matrix descriptor of a K-major, 128B-swizzled bf16 operand: rows of 128 bytes,
+// 8-row groups 1024 bytes apart (stride byte offset), version 1, layout type SWIZZLE_128B.
+__device__ inline uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                  // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset
+  d |= (uint64_t)1 << 46;                  // descriptor version
+  d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
+  return d;
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = N = 128.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate) : "memory");
+}
+__device__ inline void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this warp's 32 TMEM lanes.
+__device__ inline void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ inline float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Smem {
+  // operand tiles first (1024-byte aligned for the 128B swizzle)
+  static constexpr uint32_t kKr = 0, kVr = kTileBytes, kStage0 = 2 * kTileBytes;   // stage: K then V
+  static constexpr uint32_t kTilesEnd = 6 * kTileBytes;
+};
+
+template <bool kCenter>
+__global__ void __launch_bounds__(kThreads, 1)
+walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const CallStat* __restrict__ stats,
+               const float* __restrict__ tok_shift, int8_t* __restrict__ eta_out, int8_t* __restrict__ dbg_eta,
+               float* __restrict__ dbg_S, float* __restrict__ dbg_p, unsigned long long* __restrict__ fail_count,
+               int* __restrict__ status, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int t = G.t, P = t / kTile;
+  float* etas = reinterpret_cast<float*>(sm + Smem::kTilesEnd);          // [t] signs scaled by 1/r_value^2
+  int8_t* eta8 = reinterpret_cast<int8_t*>(etas + t);                     // [t] signs
+  uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
+  uint64_t* row_full = bars + 0;
+  uint64_t* row_empty = bars + 1;
+  uint64_t* col_full = bars + 2;     // [2]
+  uint64_t* col_empty = bars + 4;    // [2]
+  uint64_t* tmem_full = bars + 6;    // [2]
+  uint64_t* tmem_empty = bars + 8;   // [2]
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 10);
+  int* progress = reinterpret_cast<int*>(tmem_ptr_s + 1);
+  int* abort_flag = progress + 1;
+
+  const int call = blockIdx.x;
+  const CallDesc C = calls[call];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    mbar_init(row_full, 1); mbar_init(row_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(col_full + i, 1); mbar_init(col_empty + i, 1);
+      mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 128);
+    }
+    *progress = 0; *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_ptr_s)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_s;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int col_it = 0;
+      bool ok = true;
+      for (int r = 0; r < P && ok; ++r) {
+        if (!(ok = wait_bar(row_empty, (uint32_t)((r & 1) ^ 1), abort_flag))) break;
+        const int y = (int)(C.src_row + (int64_t)r * kTile);
+        mbar_expect_tx(row_full, 2 * kTileBytes);
+        tma_load_2d(sm + Smem::kKr, &tmK, 0, y, row_full);
+        tma_load_2d(sm + Smem::kKr + kHalfBytes, &tmK, 64, y, row_full);
+        tma_load_2d(sm + Smem::kVr, &tmV, 0, y, row_full);
+        tma_load_2d(sm + Smem::kVr + kHalfBytes, &tmV, 64, y, row_full);
+        for (int c = 0; c < r; ++c, ++col_it) {
+          const int s = col_it & 1;
+          if (!(ok = wait_bar(col_empty + s, (uint32_t)(((col_it >> 1) & 1) ^ 1), abort_flag))) break;
+          unsigned char* st = sm + Smem::kStage0 + (uint32_t)s * 2 * kTileBytes;
+          const int yc = (int)(C.src_row + (int64_t)c * kTile);
+          mbar_expect_tx(col_full + s, 2 * kTileBytes);
+          tma_load_2d(st, &tmK, 0, yc, col_full + s);
+          tma_load_2d(st + kHalfBytes, &tmK, 64, yc, col_full + s);
+          tma_load_2d(st + kTileBytes, &tmV, 0, yc, col_full + s);
+          tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, yc, col_full + s);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int tile_it = 0, col_it = 0;
+      bool ok = true;
+      const uint32_t kr = smem_u32(sm + Smem::kKr), vr = smem_u32(sm + Smem::kVr);
+      for (int r = 0; r < P && ok; ++r) {
+        if (!(ok = wait_bar(row_full, (uint32_t)(r & 1), abort_flag))) break;
+        for (int c = 0; c <= r; ++c, ++tile_it) {
+          const int buf = tile_it & 1;
+          if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((tile_it >> 1) & 1) ^ 1), abort_flag))) break;
+          uint32_t kb = kr, vb = vr;
+          const int s = col_it & 1;
+          if (c < r) {
+            if (!(ok = wait_bar(col_full + s, (uint32_t)((col_it >> 1) & 1), abort_flag))) break;
+            kb = smem_u32(sm + Smem::kStage0 + (uint32_t)s * 2 * kTileBytes);
+            vb = kb + kTileBytes;
+          }
+          tc_fence_after();
+          const uint32_t dK = tmem_base + (uint32_t)buf * 256u, dV = dK + 128u;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+            umma_bf16(dK, umma_desc(kr + off), umma_desc(kb + off), kk > 0);
+          }
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+            umma_bf16(dV, umma_desc(vr + off), umma_desc(vb + off), kk > 0);
+          }
+          if (c < r) { umma_commit(col_empty + s); ++col_it; }
+          else umma_commit(row_empty);
+          umma_commit(tmem_full + buf);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue + walk (warps 0-3)
+    const int head = C.stream % G.H;
+    const int layer = (C.stream / G.H) % G.L;
+    const int seq = C.stream / (G.H * G.L);
+    const float rk2 = G.fixed_rk2 > 0.f ? G.fixed_rk2 : stats[call].rk2;
+    const float rv2 = G.fixed_rv2 > 0.f ? G.fixed_rv2 : stats[call].rv2;
+    const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
+    const float scale = 1.4426950408889634f * G.inv_sqrt_d;
+    const float cw = G.c;
+    const int q = warp;                       // quarter of the panel = TMEM lane quadrant
+    const uint32_t lane_base = (uint32_t)(32 * q) << 16;
+    const float* shift = kCenter ? tok_shift + (size_t)call * t : nullptr;
+    int tile_it = 0, fails = 0;
+    bool ok = true;
+    for (int r = 0; r < P && ok; ++r) {
+      const int j = r * kTile + 32 * q + lane;          // this thread's token
+      const float u = walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, j);
+      const float thr = cw * (1.0f - 2.0f * u);
+      float nb = -rk2 * scale;                          // exponent offset of this row
+      if constexpr (kCenter) nb -= shift[j] * scale;
+      float acc = 0.f;
+      for (int c = 0; c < r && ok; ++c, ++tile_it) {
+        const int buf = tile_it & 1;
+        if (!(ok = wait_progress(progress, 4 * c + 4, abort_flag))) break;     // signs of panel c are final
+        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+        tc_fence_after();
+        const uint32_t tK = tmem_base + lane_base + (uint32_t)buf * 256u, tV = tK + 128u;
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          float dk[32], dv[32];
+          tmem_ld32(tK + ch * 32, dk);
+          tmem_ld32(tV + ch * 32, dv);
+          tmem_ld_wait();
+          const float4* e4 = reinterpret_cast<const float4*>(etas + c * kTile + ch * 32);
+#pragma unroll
+          for (int x = 0; x < 8; ++x) {
+            const float4 e = e4[x];
+            const float ev[4] = {e.x, e.y, e.z, e.w};
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+              const int i = 4 * x + y;
+              float ex = fmaf(dk[i], scale, nb);
+              if constexpr (kCenter) ex -= shift[c * kTile + ch * 32 + i] * scale;
+              acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(tmem_empty + buf);
+      }
+      if (!ok) break;
+      // ---- diagonal tile: Ghat of this row against the panel's earlier columns, then the walk
+      {
+        const int buf = tile_it & 1;
+        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+        tc_fence_after();
+        const uint32_t tK = tmem_base + lane_base + (uint32_t)buf * 256u, tV = tK + 128u;
+        float g[kTile];
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          if (ch <= q) {                                   // warp-uniform
+            float dk[32], dv[32];
+            tmem_ld32(tK + ch * 32, dk);
+            tmem_ld32(tV + ch * 32, dv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              float ex = fmaf(dk[i], scale, nb);
+              if constexpr (kCenter) ex -= shift[r * kTile + ch * 32 + i] * scale;
+              const float val = fast_exp2(ex) * dv[i];
+              g[ch * 32 + i] = (ch < q || i < lane) ? val : 0.f;   // strictly earlier tokens only
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(tmem_empty + buf);                     // TMEM buffer is free while we walk
+        ++tile_it;
+        float S = acc;
+#pragma unroll
+        for (int gi = 0; gi < 3; ++gi) {
+          if (gi < q) {                                    // warp-uniform
+            if (!(ok = wait_progress(progress, 4 * r + gi + 1, abort_flag))) break;
+            const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + gi * 32);
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+              const float4 e = e4[x];
+              s0 = fmaf(g[gi * 32 + 4 * x + 0], e.x, s0);
+              s1 = fmaf(g[gi * 32 + 4 * x + 1], e.y, s1);
+              s2 = fmaf(g[gi * 32 + 4 * x + 2], e.z, s2);
+              s3 = fmaf(g[gi * 32 + 4 * x + 3], e.w, s3);
+            }
+            S += (s0 + s1) + (s2 + s3);
+          }
+        }
+        if (!ok) break;
+        // the sequential walk over this warp's 32 tokens
+        float own[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          own[i] = 0.f;
+#pragma unroll
+          for (int qq = 0; qq < 4; ++qq)
+            if (qq == q) own[i] = g[qq * 32 + i];          // warp-uniform select of the own block
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float dec = S < thr ? inv_rv2 : -inv_rv2;
+          const float ei = __shfl_sync(0xffffffffu, dec, i);
+          S = fmaf(ei, own[i], S);                         // own[i] = 0 once this lane's token is decided
+        }
+        const bool plus = S < thr;
+        etas[j] = plus ? inv_rv2 : -inv_rv2;
+        eta8[j] = plus ? 1 : -1;
+        if (fabsf(S) > cw) ++fails;                        // FAIL of Algorithm 2: counted; the decision is the clamped one
+        if (C.dbg_off >= 0) {
+          dbg_S[C.dbg_off + j] = S;
+          dbg_p[C.dbg_off + j] = 0.5f - fminf(fmaxf(S, -cw), cw) / (2.0f * cw);
+        }
+        __syncwarp();
+        if (lane == 0) st_release(progress, 4 * r + q + 1);
+      }
+    }
+    fails = (int)__reduce_add_sync(0xffffffffu, (unsigned)fails);
+    if (lane == 0 && fails) atomicAdd(fail_count, (unsigned long long)fails);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (*abort_flag) {
+    if (tid == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
+  } else {
+    for (int i = tid; i < t; i += kThreads) {
+      const int8_t e = eta8[i];
+      eta_out[(size_t)call * t + i] = e;
+      if (C.dbg_off >= 0) dbg_eta[C.dbg_off + i] = e;
+    }
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 128; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+bool walk_tc_supported(const Geom& G) {
+  return G.is_bf16 && G.d == 128 && G.t % kTile == 0 && tc_smem_bytes(G.t) <= (size_t)227 * 1024;
+}
+
+// Encodes the two tensor maps (K and V arenas viewed as [total_rows, 128] bf16, boxes of
+// 64 columns x 128 rows, 128-byte swizzle).
+cudaError_t walk_tc_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** tmaps_out) {
+  *tmaps_out = nullptr;
+  if (!walk_tc_supported(G)) return cudaErrorNotSupported;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+  TensorMaps* tm = new TensorMaps();
+  const cuuint64_t dims[2] = {(cuuint64_t)G.d, (cuuint64_t)total_rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)G.d * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+  const cuuint32_t estr[2] = {1, 1};
+  void* bases[2] = {A.K, A.V};
+  CUtensorMap* maps[2] = {&tm->k, &tm->v};
+  for (int i = 0; i < 2; ++i) {
+    CUresult r = encode(maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[i], dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { delete tm; return cudaErrorInvalidValue; }
+  }
+  e = cudaFuncSetAttribute(walk_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(G.t));
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(walk_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(G.t));
+  if (e != cudaSuccess) { delete tm; return e; }
+  *tmaps_out = tm;
+  return cudaSuccess;
+}
+
+void walk_tc_release(void* tmaps) { delete static_cast<TensorMaps*>(tmaps); }
+
+cudaError_t launch_walk_tc(const Geom& G, const Arena& A, const CallDesc* calls, int n_calls, int level,
+                           const CallStat* stats, const float* tok_shift, int8_t* eta, int8_t* dbg_eta,
+                           float* dbg_S, float* dbg_p, unsigned long long* fail_count, int* status,
+                           const void* tmaps, const void*, cudaStream_t st) {
+  (void)A;
+  if (n_calls <= 0) return cudaSuccess;
+  if (!tmaps) return cudaErrorInvalidValue;
+  const TensorMaps* tm = static_cast<const TensorMaps*>(tmaps);
+  const size_t smem = tc_smem_bytes(G.t);
+  if (G.center_keys)
+    walk_tc_kernel<true><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
+                                                          fail_count, status, tm->k, tm->v);
+  else
+    walk_tc_kernel<false><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
+                                                           fail_count, status, tm->k, tm->v);
+  return cudaGetLastError();
 }
 
 }  // namespace bkv

@@ -48,11 +48,12 @@ def test_tiny_single_head_fp32(cuda_lib):
 
 
 @pytest.mark.parametrize("dtype,d,t,T,gram", [("fp32", 128, 256, 2, 1), ("bf16", 128, 256, 2, 1), ("bf16", 64, 128, 3, 1),
-                                              ("fp32", 64, 64, 1, 1)])
+                                              ("fp32", 64, 64, 1, 1), ("bf16", 128, 128, 1, 2), ("bf16", 128, 256, 2, 2),
+                                              ("bf16", 128, 1024, 2, 2)])
 def test_aggressive_walk_exercises_the_gram_arithmetic(cuda_lib, dtype, d, t, T, gram):
     """Small c and small keys make p_j stray far from 1/2, so S_j parity tests every Gram entry."""
     B, L, H, g = 1, 2, 2, 4
-    n = t * 8 + 37
+    n = t * (8 if t < 1024 else 4) + 37
     K, V = _layer_inputs("llama", 77, B, L, H, n, d, dtype, key_scale=0.06)
     hz = Harness(cuda_lib, B=B, L=L, H=H, g=g, d=d, dtype=dtype, t=t, T=T, N=n, seed=3, c_override=0.75, gram_path=gram)
     for l in range(L):
@@ -178,12 +179,14 @@ def test_per_stream_append_ragged_lengths_and_errors(cuda_lib):
         bk.Context(head_dim=96)
 
 
-def test_key_centering_flag(cuda_lib):
+@pytest.mark.parametrize("gram", [1, 2])
+def test_key_centering_flag(cuda_lib, gram):
     B, L, H, g, d, t = 1, 1, 2, 1, 128, 128
     n = t * 4
     K, V = _layer_inputs("llama", 41, B, L, H, n, d, "bf16", key_scale=0.06)
     K = synth.round_to(K + 1.5, "bf16")       # a large common offset that centering removes
-    hz = Harness(cuda_lib, B=B, L=L, H=H, g=g, d=d, dtype="bf16", t=t, T=1, N=n, seed=2, c_override=0.75, center_keys=1)
+    hz = Harness(cuda_lib, B=B, L=L, H=H, g=g, d=d, dtype="bf16", t=t, T=1, N=n, seed=2, c_override=0.75, center_keys=1,
+                 gram_path=gram)
     hz.append_layer(0, K[:, 0], V[:, 0])
     hz.compress()
     hz.check_all(5e-4)
