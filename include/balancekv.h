@@ -118,6 +118,32 @@ int balancekv_decode_attn(balancekv_ctx* ctx, int layer, const void* q, void* ou
 int balancekv_decode_attn_host(balancekv_ctx* ctx, int layer, const void* q_host, void* out_host,
                                void* stream);
 
+/* Decode attention for callers that must not allocate (the paper has no counterpart: this
+ * is a deployment variant of balancekv_decode_attn, not a step of the method).
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a serving loop that
+ * cannot afford cudaMalloc's device-wide synchronisation, a plugin that only ever receives
+ * buffers from its host framework, a process whose memory pool is fully committed.  Such a
+ * caller cannot create a context (that allocates the cache), so it keeps the cache rows
+ * itself and passes them in:
+ *   K, V : [n_streams, cache_len, head_dim]   q, out : [n_streams, group, head_dim]
+ * (device pointers, 16-byte aligned, dtype 0 = float32 / 1 = bfloat16).  In every stream the
+ * first n_heavy rows carry weight 2^level and the remaining rows weight 1; out is
+ * sum_i w_i e^{<k_i,q>/sqrt d} v_i / sum_i w_i e^{<k_i,q>/sqrt d}, the same arithmetic as
+ * balancekv_decode_attn.
+ *
+ * The split-K scratch is a fixed 8 MiB array inside the library image (held by every GPU
+ * that loads the library, until the process exits); the call performs no cudaMalloc, cudaFree
+ * or other allocating call.  A problem whose scratch (about n_streams * splits * group *
+ * (head_dim+2) * 4 bytes, splits <= 64) exceeds the array is rejected with BALANCEKV_E_NOMEM
+ * and a message on stderr.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.  All calls share
+ * the array: the part a call uses is re-initialised by the call itself, but two calls that
+ * overlap on the GPU (different CUDA streams) race on it -- issue them on one stream. */
+int balancekv_decode_attn_static(const void* K, const void* V, int n_streams, int cache_len, int n_heavy,
+                                 int level, const void* q, void* out, int group, int head_dim, int dtype,
+                                 void* stream);
+
 /* Load an already-compressed set into level `level` of every stream of one layer
  * (weight 2^level, the weights of Theorem 3.3's estimator): K, V: [n_seqs, n_kv_heads,
  * n_tokens, head_dim]; orig_idx (may be NULL): [n_seqs, n_kv_heads, n_tokens] original

@@ -5,6 +5,7 @@ from .binding import (  # noqa: E402,F401
     Context,
     EXPORTS,
     LIB_PATH,
+    decode_attn_static,
     load,
     plan_calls,
 )

@@ -21,7 +21,7 @@ EXPORTS = [
     "balancekv_decode_attn", "balancekv_decode_attn_host", "balancekv_cache_load_level",
     "balancekv_cache_view", "balancekv_level_sizes", "balancekv_debug_enable", "balancekv_debug_call",
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
-    "balancekv_profile_enable", "balancekv_profile_read",
+    "balancekv_profile_enable", "balancekv_profile_read", "balancekv_decode_attn_static",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -83,6 +83,7 @@ def load():
     lib.balancekv_reset.argtypes = [vp, vp]
     lib.balancekv_profile_enable.argtypes = [vp, ci]
     lib.balancekv_profile_read.argtypes = [vp, vp]
+    lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     for name in EXPORTS:
         if name != "balancekv_strerror":
             getattr(lib, name).restype = ci
@@ -270,6 +271,26 @@ class Context:
         s = Stats()
         _check(self.lib.balancekv_stats(self._h, C.byref(s)), "balancekv_stats")
         return {n: getattr(s, n) for n, _ in Stats._fields_}
+
+
+def decode_attn_static(K, V, n_heavy, level, q, out=None, stream=None):
+    """Allocation-free decode attention over caller-owned caches (see balancekv.h).
+
+    K, V: CUDA tensors [n_streams, cache_len, d]; q: [n_streams, group, d]; the first
+    ``n_heavy`` rows of every stream weigh 2**level, the rest 1.  ``out`` must be supplied by
+    callers that may not allocate; when it is None a tensor is created for convenience."""
+    import torch
+
+    assert K.is_cuda and V.is_cuda and q.is_cuda and K.is_contiguous() and V.is_contiguous() and q.is_contiguous()
+    assert K.shape == V.shape and K.dtype == V.dtype == q.dtype and q.shape[0] == K.shape[0] and q.shape[2] == K.shape[2]
+    if out is None:
+        out = torch.empty_like(q)
+    dtype_code = {torch.float32: 0, torch.bfloat16: 1}[K.dtype]
+    _check(load().balancekv_decode_attn_static(C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()), K.shape[0],
+                                               K.shape[1], n_heavy, level, C.c_void_p(q.data_ptr()),
+                                               C.c_void_p(out.data_ptr()), q.shape[1], K.shape[2], dtype_code,
+                                               _stream_ptr(stream)), "balancekv_decode_attn_static")
+    return out
 
 
 class _RawDevice:
