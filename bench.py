@@ -206,6 +206,10 @@ def main():
     ctx = bk.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, head_dim=d, dtype="bf16", block=t, levels=T,
                      max_tokens=n_ctx + n_dec, seed=w["walk_seed"] + rank, gram_path=args.gram_path)
 
+    raw_stream = int(torch.cuda.current_stream().cuda_stream)
+    q_list, K_list, V_list = list(q_d.unbind(0)), list(K_dec.unbind(0)), list(V_dec.unbind(0))
+    qh_list, Kh_list, Vh_list, oh_list = list(q_h.unbind(0)), list(K_dec_h.unbind(0)), list(V_dec_h.unbind(0)), list(out_h.unbind(0))
+
     def step_device(ev=None):
         ctx.reset()
         if ev: ev[0].record()
@@ -213,8 +217,7 @@ def main():
         ctx.compress()
         if ev: ev[1].record()
         for s in range(n_dec):
-            ctx.stream_append_layer(0, K_dec[s], V_dec[s])
-            ctx.decode_attn(0, q_d[s], out_d)
+            ctx.stream_step(0, q_list[s], K_list[s], V_list[s], out_d, stream=raw_stream)
         if ev: ev[2].record()
 
     def step_host():
@@ -222,8 +225,7 @@ def main():
         ctx.stream_append_layer_host(0, K_ctx_h, V_ctx_h)
         ctx.compress()
         for s in range(n_dec):
-            ctx.stream_append_layer_host(0, K_dec_h[s], V_dec_h[s])
-            ctx.decode_attn_host(0, q_h[s], out_h[s])
+            ctx.stream_step_host(0, qh_list[s], Kh_list[s], Vh_list[s], oh_list[s], stream=raw_stream)
 
     def barrier():
         if world > 1:
@@ -303,7 +305,7 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        sample, dsteps = n_ctx // 8, max(n_dec // 8, 1) if n_dec else 0
+        sample, dsteps = n_ctx, (max(n_dec // 8, 1) if n_dec else 0)
         dt, units, threads = oracle_sample(w, Kf, Vf, qf, sample, dsteps)
         cpu = dict(value=units / dt, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
                    sample=f"first {sample} of {n_ctx} context tokens of each of the {B * H} streams + {dsteps} decode steps")

@@ -113,6 +113,17 @@ int balancekv_compress_layer(balancekv_ctx* ctx, int layer, int T, void* stream)
  * head_dim] in the context's dtype.  With T = 0 this is Eq. (1) exactly. */
 int balancekv_decode_attn(balancekv_ctx* ctx, int layer, const void* q, void* out, void* stream);
 
+/* One step of the streaming problem of Section 2.1: the triple (q_j, k_j, v_j) of every
+ * stream of a layer arrives, k_j, v_j join C^0 (Algorithm 3; decode-phase tokens stay
+ * uncompressed until a later compress), and z_j is returned.  k_new, v_new: [n_seqs,
+ * n_kv_heads, head_dim]; q, out as in balancekv_decode_attn.  Equivalent to
+ * balancekv_stream_append_layer(.., 1) followed by balancekv_decode_attn. */
+int balancekv_stream_step(balancekv_ctx* ctx, int layer, const void* q, const void* k_new, const void* v_new,
+                          void* out, void* stream);
+/* Same with HOST buffers for q, k_new, v_new and out (see the other *_host calls). */
+int balancekv_stream_step_host(balancekv_ctx* ctx, int layer, const void* q_host, const void* k_host,
+                               const void* v_host, void* out_host, void* stream);
+
 /* As above with HOST q and out: q is copied in, out copied back, both on `stream`;
  * the call returns without synchronising (synchronise the stream before reading out). */
 int balancekv_decode_attn_host(balancekv_ctx* ctx, int layer, const void* q_host, void* out_host,

@@ -22,6 +22,7 @@ EXPORTS = [
     "balancekv_cache_view", "balancekv_level_sizes", "balancekv_debug_enable", "balancekv_debug_call",
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
     "balancekv_profile_enable", "balancekv_profile_read", "balancekv_decode_attn_static",
+    "balancekv_stream_step", "balancekv_stream_step_host",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -81,6 +82,8 @@ def load():
     lib.balancekv_strerror.restype = C.c_char_p
     lib.balancekv_plan_calls.argtypes = [ci, ci, ci, vp, ci, vp, ci]
     lib.balancekv_reset.argtypes = [vp, vp]
+    lib.balancekv_stream_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
+    lib.balancekv_stream_step_host.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.balancekv_profile_enable.argtypes = [vp, ci]
     lib.balancekv_profile_read.argtypes = [vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
@@ -99,6 +102,8 @@ def _check(code: int, what: str):
 def _stream_ptr(stream):
     import torch
 
+    if isinstance(stream, int):          # a raw cudaStream_t
+        return C.c_void_p(stream)
     s = stream if stream is not None else torch.cuda.current_stream()
     return C.c_void_p(s.cuda_stream)
 
@@ -198,6 +203,20 @@ class Context:
         _check(self.lib.balancekv_decode_attn(self._h, layer, self._dev(q, "q"), self._dev(out, "out"),
                                               _stream_ptr(stream)), "balancekv_decode_attn")
         return out
+
+    def stream_step(self, layer, q, k_new, v_new, out, stream=None):
+        """Append one token per stream of the layer and decode: q, out [B, Hq, d]; k_new, v_new [B, H, d]."""
+        _check(self.lib.balancekv_stream_step(self._h, layer, self._dev(q, "q"), self._dev(k_new, "k_new"),
+                                              self._dev(v_new, "v_new"), self._dev(out, "out"), _stream_ptr(stream)),
+               "balancekv_stream_step")
+        return out
+
+    def stream_step_host(self, layer, q_host, k_host, v_host, out_host, stream=None):
+        _check(self.lib.balancekv_stream_step_host(self._h, layer, C.c_void_p(q_host.data_ptr()),
+                                                   C.c_void_p(k_host.data_ptr()), C.c_void_p(v_host.data_ptr()),
+                                                   C.c_void_p(out_host.data_ptr()), _stream_ptr(stream)),
+               "balancekv_stream_step_host")
+        return out_host
 
     def decode_attn_host(self, layer, q_host, out_host, stream=None):
         assert not q_host.is_cuda and not out_host.is_cuda and q_host.dtype == self.dtype

@@ -83,6 +83,7 @@ struct balancekv_ctx {
   void* bounce_out = nullptr;
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
+  std::vector<std::vector<int>> layer_stream_ids;
 
   // optional per-class kernel timing
   bool profiling = false;
@@ -317,7 +318,7 @@ int balancekv_destroy(balancekv_ctx* c) {
 // Appends (level 0) or loads (level T) n rows per listed stream from a caller tensor laid
 // out as consecutive [n, d] blocks in the order of `streams`.
 static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int level, const void* K, const void* V,
-                       const int32_t* idx, int n, cudaStream_t st) {
+                       const int32_t* idx, int n, cudaStream_t st, int whole_layer = -1) {
   if (!K || !V || n < 0) return BALANCEKV_E_INVAL;
   if (!aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
   if (n == 0) return BALANCEKV_OK;
@@ -333,6 +334,29 @@ static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int le
       if ((int64_t)S.start0 + S.len0 + n > Lo.cap0) return BALANCEKV_E_NOMEM;
     } else {
       if ((int64_t)S.lvl_len[T] + n > Lo.capT) return BALANCEKV_E_NOMEM;
+    }
+  }
+  if (whole_layer >= 0) {
+    // lockstep layer: every stream has the same fill, so the kernel derives the descriptors
+    const StreamState& S0 = c->st[streams[0]];
+    bool same = true;
+    for (int s : streams) {
+      const StreamState& S = c->st[s];
+      same &= S.start0 == S0.start0 && S.len0 == S0.len0 && S.appended == S0.appended && S.lvl_len[T] == S0.lvl_len[T];
+    }
+    if (same) {
+      const int rel = level == 0 ? S0.start0 + S0.len0 : S0.lvl_len[T];
+      const int idx0 = level == 0 ? (int)S0.appended : S0.lvl_len[T];
+      const int new_len = (level == 0 ? S0.len0 : S0.lvl_len[T]) + n;
+      for (int s : streams) {
+        StreamState& S = c->st[s];
+        if (level == 0) { S.len0 += n; S.appended += n; S.pending += n; c->tokens_appended += n; }
+        else S.lvl_len[T] += n;
+      }
+      ProfScope ps(c, 0, st);
+      BKV_CUDA(launch_append_uniform(c->G, c->A, whole_layer, level, rel, idx0, n, new_len, K, V, idx, st));
+      c->kernels_launched++;
+      return BALANCEKV_OK;
     }
   }
   std::vector<AppendDesc> descs(streams.size());
@@ -376,16 +400,18 @@ int balancekv_stream_append(balancekv_ctx* c, int seq, int layer, int kv_head, c
   return append_impl(c, s, 0, K_blk, V_blk, nullptr, n_tokens, static_cast<cudaStream_t>(stream));
 }
 
-static std::vector<int> layer_streams(const balancekv_ctx* c, int layer) {
-  std::vector<int> v;
-  for (int s = 0; s < c->cfg.n_seqs; ++s)
-    for (int h = 0; h < c->cfg.n_kv_heads; ++h) v.push_back(stream_id(c, s, layer, h));
+static const std::vector<int>& layer_streams(balancekv_ctx* c, int layer) {
+  if (c->layer_stream_ids.empty()) c->layer_stream_ids.resize(c->cfg.n_layers);
+  std::vector<int>& v = c->layer_stream_ids[layer];
+  if (v.empty())
+    for (int s = 0; s < c->cfg.n_seqs; ++s)
+      for (int h = 0; h < c->cfg.n_kv_heads; ++h) v.push_back(stream_id(c, s, layer, h));
   return v;
 }
 
 int balancekv_stream_append_layer(balancekv_ctx* c, int layer, const void* K, const void* V, int n_tokens, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
-  return append_impl(c, layer_streams(c, layer), 0, K, V, nullptr, n_tokens, static_cast<cudaStream_t>(stream));
+  return append_impl(c, layer_streams(c, layer), 0, K, V, nullptr, n_tokens, static_cast<cudaStream_t>(stream), layer);
 }
 
 int balancekv_stream_append_layer_host(balancekv_ctx* c, int layer, const void* K_host, const void* V_host,
@@ -404,14 +430,14 @@ int balancekv_stream_append_layer_host(balancekv_ctx* c, int layer, const void* 
   }
   BKV_CUDA(cudaMemcpyAsync(c->bounce_K, K_host, bytes, cudaMemcpyHostToDevice, st));
   BKV_CUDA(cudaMemcpyAsync(c->bounce_V, V_host, bytes, cudaMemcpyHostToDevice, st));
-  return append_impl(c, layer_streams(c, layer), 0, c->bounce_K, c->bounce_V, nullptr, n_tokens, st);
+  return append_impl(c, layer_streams(c, layer), 0, c->bounce_K, c->bounce_V, nullptr, n_tokens, st, layer);
 }
 
 int balancekv_cache_load_level(balancekv_ctx* c, int layer, int level, const void* K, const void* V,
                                const int32_t* orig_idx, int n_tokens, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
   if (level != 0 && level != c->cfg.levels) return BALANCEKV_E_INVAL;
-  return append_impl(c, layer_streams(c, layer), level, K, V, orig_idx, n_tokens, static_cast<cudaStream_t>(stream));
+  return append_impl(c, layer_streams(c, layer), level, K, V, orig_idx, n_tokens, static_cast<cudaStream_t>(stream), layer);
 }
 
 // Runs one planned batch: per level radii -> walk -> selection/compaction, then the
@@ -549,6 +575,20 @@ int balancekv_decode_attn_host(balancekv_ctx* c, int layer, const void* q_host, 
   if (rc) return rc;
   BKV_CUDA(cudaMemcpyAsync(out_host, c->bounce_out, bytes, cudaMemcpyDeviceToHost, st));
   return BALANCEKV_OK;
+}
+
+int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                          void* stream) {
+  int rc = balancekv_stream_append_layer(c, layer, k_new, v_new, 1, stream);
+  if (rc) return rc;
+  return balancekv_decode_attn(c, layer, q, out, stream);
+}
+
+int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, const void* k_host, const void* v_host,
+                               void* out_host, void* stream) {
+  int rc = balancekv_stream_append_layer_host(c, layer, k_host, v_host, 1, stream);
+  if (rc) return rc;
+  return balancekv_decode_attn_host(c, layer, q_host, out_host, stream);
 }
 
 int balancekv_level_sizes(balancekv_ctx* c, int seq, int layer, int kv_head, int32_t* sizes) {

@@ -134,6 +134,9 @@ struct Arena {
 
 cudaError_t launch_append(const Geom& G, const Arena& A, const AppendDesc* descs, int n_desc, int max_rows,
                           const void* Ksrc, const void* Vsrc, const int32_t* idx_src, cudaStream_t st);
+cudaError_t launch_append_uniform(const Geom& G, const Arena& A, int layer, int level, int rel_row, int idx0, int n,
+                                  int new_len, const void* Ksrc, const void* Vsrc, const int32_t* idx_src,
+                                  cudaStream_t st);
 cudaError_t launch_move(const Geom& G, const Arena& A, const MoveDesc* descs, int n_desc, int max_rows,
                         cudaStream_t st);
 cudaError_t launch_radii(const Geom& G, const Arena& A, const CallDesc* calls, int n_calls, CallStat* stats,

@@ -323,8 +323,12 @@ cudaError_t launch_t(const Geom& G, const Arena& A, int layer, const void* q, vo
                      int splits, int* status, cudaStream_t st) {
   auto kern = decode_kernel<kBf16, D, GQ>;
   const size_t smem = (size_t)kStages * 2 * kTileBytes + kStages * sizeof(uint64_t);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  static bool configured = false;   // one device per process uses this library
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
   const int n_sl = G.B * G.H;
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;

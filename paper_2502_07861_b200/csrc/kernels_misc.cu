@@ -37,6 +37,31 @@ append_kernel(Geom G, Arena A, const AppendDesc* __restrict__ descs, const void*
   if (blockIdx.y == 0 && threadIdx.x == 0) A.seg[(size_t)D.stream * (G.T + 1) + D.level].len = D.new_len;
 }
 
+// Append for a layer whose streams are in lockstep (same level-0 fill): the per-stream
+// descriptor is implied by the block index, so no descriptor array travels to the device.
+__global__ void __launch_bounds__(256)
+append_uniform_kernel(Geom G, Arena A, int layer, int level, int rel_row, int idx0, int n, int new_len,
+                      const void* __restrict__ Ksrc, const void* __restrict__ Vsrc, const int32_t* __restrict__ idx_src) {
+  const int sl = blockIdx.x;                                 // seq * H + head
+  const int stream = ((sl / G.H) * G.L + layer) * G.H + (sl % G.H);
+  const int64_t dst_row = (int64_t)stream * G.rows_per_stream + G.region_off[level] + rel_row;
+  const int row0 = blockIdx.y * kCopyRows;
+  if (row0 < n) {
+    const int rows = min(kCopyRows, n - row0);
+    const int esz = G.is_bf16 ? 2 : 4;
+    const int chunks = G.d * esz / 16;
+    const size_t dst_b = (size_t)(dst_row + row0) * G.d * esz;
+    const size_t src_b = ((size_t)sl * n + row0) * G.d * esz;
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(Ksrc) + src_b), rows, chunks);
+    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
+              reinterpret_cast<const uint4*>(static_cast<const char*>(Vsrc) + src_b), rows, chunks);
+    for (int i = threadIdx.x; i < rows; i += blockDim.x)
+      A.idx[dst_row + row0 + i] = idx_src ? idx_src[(size_t)sl * n + row0 + i] : idx0 + row0 + i;
+  }
+  if (blockIdx.y == 0 && threadIdx.x == 0) A.seg[(size_t)stream * (G.T + 1) + level].len = new_len;
+}
+
 __global__ void __launch_bounds__(256)
 move_kernel(Geom G, Arena A, const MoveDesc* __restrict__ descs) {
   const MoveDesc D = descs[blockIdx.x];
@@ -140,6 +165,14 @@ cudaError_t launch_append(const Geom& G, const Arena& A, const AppendDesc* descs
   dim3 grid(n_desc, (max_rows + kCopyRows - 1) / kCopyRows);
   if (grid.y == 0) grid.y = 1;
   append_kernel<<<grid, 256, 0, st>>>(G, A, descs, Ksrc, Vsrc, idx_src);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append_uniform(const Geom& G, const Arena& A, int layer, int level, int rel_row, int idx0, int n,
+                                  int new_len, const void* Ksrc, const void* Vsrc, const int32_t* idx_src,
+                                  cudaStream_t st) {
+  dim3 grid(G.B * G.H, (n + kCopyRows - 1) / kCopyRows);
+  append_uniform_kernel<<<grid, n >= 16 ? 256 : 64, 0, st>>>(G, A, layer, level, rel_row, idx0, n, new_len, Ksrc, Vsrc, idx_src);
   return cudaGetLastError();
 }
 

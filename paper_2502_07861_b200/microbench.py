@@ -1,0 +1,141 @@
+"""Kernel-level timing of the BalanceKV library on synthetic device data.
+
+    python -m paper_2502_07861_b200.microbench decode   --batch 32 --cache-len 8192 --levels 2
+    python -m paper_2502_07861_b200.microbench compress --streams 8 --context 32768 --block 1024 --levels 2
+
+Prints one JSON line per run.  Inputs are drawn on the device (torch.randn), which is enough
+for timing; parity is the tests' job.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import torch
+
+from . import binding as bk
+
+_ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peaks():
+    p = os.path.join(_ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return float(j["hbm_gbs"]), float(j["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def run_decode(a):
+    """Decode attention over caches loaded directly at level T (the decode-sweep shape)."""
+    B, H, g, d, Lc, T = a.batch, a.kv_heads, a.group, a.head_dim, a.cache_len, a.levels
+    esz = 2
+    bytes_layer = B * H * Lc * 2 * d * esz
+    # enough distinct layers that a layer is evicted from L2 (126 MB) before it is read again
+    n_layers = max(2, min(a.max_layers, (512 << 20) // max(bytes_layer, 1) + 1))
+    ctx = bk.Context(n_seqs=B, n_layers=n_layers, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64,
+                     levels=T, max_tokens=Lc << T)
+    K = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    V = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    for l in range(n_layers):
+        ctx.cache_load_level(l, T, K, V)
+    q = torch.randn(B, H * g, d, device="cuda").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    raw = int(torch.cuda.current_stream().cuda_stream)
+    for i in range(3 * n_layers):
+        ctx.decode_attn(i % n_layers, q, out, stream=raw)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    iters = a.iters
+    e0.record()
+    for i in range(iters):
+        ctx.decode_attn(i % n_layers, q, out, stream=raw)
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / iters
+    hbm, _, src = _peaks()
+    gbs = bytes_layer / (us * 1e-6) / 1e9
+    st = ctx.stats()
+    print(json.dumps(dict(kernel="decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
+                          layers_cycled=n_layers, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
+                          peak_gbs=hbm, frac=gbs / hbm, peak_source=src, device_status=st["device_status"])))
+    ctx.close()
+
+
+def run_compress(a):
+    """append + compress of `streams` streams (one layer), timed per kernel class."""
+    S, d, n, t, T = a.streams, a.head_dim, a.context, a.block, a.levels
+    ctx = bk.Context(n_seqs=1, n_layers=1, n_kv_heads=S, n_q_heads=S, head_dim=d, dtype="bf16", block=t, levels=T,
+                     max_tokens=n, gram_path=a.gram_path, c_override=a.c_override)
+    K = torch.randn(1, S, n, d, device="cuda", dtype=torch.float32)
+    if a.outliers:
+        K[..., :4] *= 10.0
+    K = K.to(torch.bfloat16)
+    V = torch.randn(1, S, n, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        ctx.reset(); ctx.stream_append_layer(0, K, V); ctx.compress()
+    ctx.profile_enable(True)
+    ctx.profile_read()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tot = 0.0
+    for i in range(a.iters):
+        ctx.reset()
+        ctx.stream_append_layer(0, K, V)
+        flush.fill_(i & 255)
+        e0.record()
+        ctx.compress()
+        e1.record()
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1)
+    prof = ctx.profile_read()
+    n_calls = S * sum((n // t) >> l for l in range(T))
+    flop = n_calls * 2.0 * (t * (t - 1) / 2.0) * 2.0 * d
+    gw_n, gw_ms = prof["gram_walk"]
+    cp_n, cp_ms = prof["compact"]
+    hbm, tf, src = _peaks()
+    tfl = flop * a.iters / (gw_ms * 1e-3) / 1e12 if gw_ms else 0.0
+    cp_bytes = n_calls * ((t // 2) * (4 * d * 2 + 8) + t)
+    cp_gbs = cp_bytes * a.iters / (cp_ms * 1e-3) / 1e9 if cp_ms else 0.0
+    st = ctx.stats()
+    print(json.dumps(dict(kernel="compress", streams=S, context=n, block=t, levels=T, calls=n_calls,
+                          compress_ms=tot / a.iters, gram_walk_ms=gw_ms / a.iters, gram_walk_launches=gw_n // a.iters,
+                          gram_walk_tflops=tfl, tensor_peak=tf, tensor_frac=tfl / tf,
+                          compact_ms=cp_ms / a.iters, compact_gbs=cp_gbs, hbm_peak=hbm, compact_frac=cp_gbs / hbm,
+                          radii_ms=prof["radii"][1] / a.iters, bookkeeping_ms=prof["bookkeeping"][1] / a.iters,
+                          token_heads_per_s=S * n / (tot / a.iters * 1e-3), walk_fails=st["walk_fails"],
+                          device_status=st["device_status"], peak_source=src)))
+    ctx.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    d = sub.add_parser("decode")
+    d.add_argument("--batch", type=int, default=32)
+    d.add_argument("--kv-heads", type=int, default=8)
+    d.add_argument("--group", type=int, default=5)
+    d.add_argument("--head-dim", type=int, default=128)
+    d.add_argument("--cache-len", type=int, default=8192)
+    d.add_argument("--levels", type=int, default=2)
+    d.add_argument("--iters", type=int, default=50)
+    d.add_argument("--max-layers", type=int, default=16)
+    c = sub.add_parser("compress")
+    c.add_argument("--streams", type=int, default=8)
+    c.add_argument("--head-dim", type=int, default=128)
+    c.add_argument("--context", type=int, default=32768)
+    c.add_argument("--block", type=int, default=1024)
+    c.add_argument("--levels", type=int, default=2)
+    c.add_argument("--iters", type=int, default=10)
+    c.add_argument("--gram-path", type=int, default=0)
+    c.add_argument("--c-override", type=float, default=0.0)
+    c.add_argument("--outliers", type=int, default=1)
+    a = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("microbench needs a CUDA device")
+    (run_decode if a.cmd == "decode" else run_compress)(a)
+
+
+if __name__ == "__main__":
+    main()
