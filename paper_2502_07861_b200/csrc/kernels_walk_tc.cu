@@ -5,15 +5,18 @@
 // is visited in 128 x 128 tiles of its lower triangle, row panel by row panel.  For a tile,
 // TMA brings the bf16 rows of K and V into 128B-swizzled shared memory, one thread issues
 // tcgen05.mma (bf16 x bf16 -> fp32) for K_r K_c^T and V_r V_c^T into two TMEM accumulators,
-// and an epilogue warpgroup (thread = row) reads them back with tcgen05.ld, applies
-// exp2/scale/product and folds the tile into the row's running correlation
+// and two epilogue warpgroups (thread = row, alternating tiles) read them back with tcgen05.ld,
+// apply exp2/scale/product and fold the tile into the row's running correlation
 //   S_j = sum_{i<j} eta_i Ghat_ij
-// with the signs of earlier panels.  The diagonal tile feeds the sequential walk: warp q owns
-// rows 32q..32q+31 of the panel, lane l owns one token, signs travel by warp shuffle,
+// with the signs of earlier panels.  The diagonal tile feeds the walk: warp q owns rows
+// 32q..32q+31 of the panel, lane l owns one token,
 //   eta_j = +1  iff  u_j < 1/2 - S_j/(2c)  <=>  S_j < c (1 - 2 u_j),
-// u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).
-// TMEM is double buffered (2 x 256 columns), so the tensor core works on the next tile while
-// the epilogue drains the previous one; Ghat never touches global memory.
+// u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).  Inside a 32-token
+// group the sequential recurrence is solved by sweeps (decide all tokens from the current
+// signs, repeat until nothing changes), which reaches exactly the sequential result.
+// TMEM is double buffered (2 x 256 columns, one buffer per warpgroup), so the tensor core
+// works on the next tile while an epilogue drains the previous one; Ghat never touches
+// global memory.
 //
 // Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
 // roles leave their loops, TMEM is freed and the kernel returns.
@@ -26,7 +29,8 @@ namespace bkv {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kThreads = 192;              // warps 0-3: epilogue + walk, warp 4: TMA, warp 5: MMA
+constexpr int kThreads = 320;              // warps 0-3, 4-7: two epilogue + walk warpgroups, warp 8: TMA, warp 9: MMA
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
 constexpr uint32_t kHalfBytes = 16384;     // [128 rows][64 bf16] = one swizzle-atom column of a tile
 constexpr uint32_t kTileBytes = 32768;     // [128 rows][128 bf16]
 constexpr uint32_t kTmemCols = 512;
@@ -158,7 +162,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int t = G.t, P = t / kTile;
   float* etas = reinterpret_cast<float*>(sm + Smem::kTilesEnd);          // [t] signs scaled by 1/r_value^2
-  int8_t* eta8 = reinterpret_cast<int8_t*>(etas + t);                     // [t] signs
+  float* xacc = etas + t;                                                 // [2][128] partial correlations handed over
+  int8_t* eta8 = reinterpret_cast<int8_t*>(xacc + 2 * kTile);             // [t] signs
   uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
   uint64_t* row_full = bars + 0;
   uint64_t* row_empty = bars + 1;
@@ -166,7 +171,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   uint64_t* col_empty = bars + 4;    // [2]
   uint64_t* tmem_full = bars + 6;    // [2]
   uint64_t* tmem_empty = bars + 8;   // [2]
-  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 10);
+  uint64_t* xacc_full = bars + 10;   // [2]
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 12);
   int* progress = reinterpret_cast<int*>(tmem_ptr_s + 1);
   int* abort_flag = progress + 1;
 
@@ -179,12 +185,13 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     for (int i = 0; i < 2; ++i) {
       mbar_init(col_full + i, 1); mbar_init(col_empty + i, 1);
       mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 128);
+      mbar_init(xacc_full + i, 128);
     }
     *progress = 0; *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_ptr_s)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -193,7 +200,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
 
-  if (warp == 4) {
+  if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int col_it = 0;
@@ -220,7 +227,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       }
     }
     __syncwarp();
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       int tile_it = 0, col_it = 0;
@@ -229,7 +236,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       for (int r = 0; r < P && ok; ++r) {
         if (!(ok = wait_bar(row_full, (uint32_t)(r & 1), abort_flag))) break;
         for (int c = 0; c <= r; ++c, ++tile_it) {
-          const int buf = tile_it & 1;
+          const int buf = tile_it & 1;                 // tile i belongs to epilogue warpgroup i & 1
           if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((tile_it >> 1) & 1) ^ 1), abort_flag))) break;
           uint32_t kb = kr, vb = vr;
           const int s = col_it & 1;
@@ -258,7 +265,13 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue + walk (warps 0-3)
+    // ------------------------------------------------------------------ two epilogue warpgroups
+    // Tiles are numbered in issue order; warpgroup wg drains tiles i with (i & 1) == wg from
+    // TMEM buffer wg.  Both keep a partial running correlation per row of the current panel;
+    // the group that gets the diagonal tile collects the other's partial and walks the panel.
+    const int wg = warp >> 2;
+    const int q = warp & 3;                   // quarter of the panel = TMEM lane quadrant
+    const int row = 32 * q + lane;
     const int head = C.stream % G.H;
     const int layer = (C.stream / G.H) % G.L;
     const int seq = C.stream / (G.H * G.L);
@@ -267,29 +280,25 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
     const float scale = 1.4426950408889634f * G.inv_sqrt_d;
     const float cw = G.c;
-    const int q = warp;                       // quarter of the panel = TMEM lane quadrant
-    const uint32_t lane_base = (uint32_t)(32 * q) << 16;
+    const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)wg * 256u;
     const float* shift = kCenter ? tok_shift + (size_t)call * t : nullptr;
-    int tile_it = 0, fails = 0;
+    int tile_it = 0, my_tiles = 0, fails = 0;
     bool ok = true;
     for (int r = 0; r < P && ok; ++r) {
-      const int j = r * kTile + 32 * q + lane;          // this thread's token
-      const float u = walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, j);
-      const float thr = cw * (1.0f - 2.0f * u);
-      float nb = -rk2 * scale;                          // exponent offset of this row
+      const int j = r * kTile + row;                      // this thread's token in the panel
+      float nb = -rk2 * scale;                            // exponent offset of this row
       if constexpr (kCenter) nb -= shift[j] * scale;
       float acc = 0.f;
       for (int c = 0; c < r && ok; ++c, ++tile_it) {
-        const int buf = tile_it & 1;
+        if ((tile_it & 1) != wg) continue;
         if (!(ok = wait_progress(progress, 4 * c + 4, abort_flag))) break;     // signs of panel c are final
-        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+        if (!(ok = wait_bar(tmem_full + wg, (uint32_t)(my_tiles & 1), abort_flag))) break;
         tc_fence_after();
-        const uint32_t tK = tmem_base + lane_base + (uint32_t)buf * 256u, tV = tK + 128u;
 #pragma unroll 1
         for (int ch = 0; ch < 4; ++ch) {
           float dk[32], dv[32];
-          tmem_ld32(tK + ch * 32, dk);
-          tmem_ld32(tV + ch * 32, dv);
+          tmem_ld32(tbase + ch * 32, dk);
+          tmem_ld32(tbase + 128 + ch * 32, dv);
           tmem_ld_wait();
           const float4* e4 = reinterpret_cast<const float4*>(etas + c * kTile + ch * 32);
 #pragma unroll
@@ -306,80 +315,121 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
           }
         }
         tc_fence_before();
-        mbar_arrive(tmem_empty + buf);
+        mbar_arrive(tmem_empty + wg);
+        ++my_tiles;
       }
       if (!ok) break;
-      // ---- diagonal tile: Ghat of this row against the panel's earlier columns, then the walk
-      {
-        const int buf = tile_it & 1;
-        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
-        tc_fence_after();
-        const uint32_t tK = tmem_base + lane_base + (uint32_t)buf * 256u, tV = tK + 128u;
-        float g[kTile];
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          if (ch <= q) {                                   // warp-uniform
-            float dk[32], dv[32];
-            tmem_ld32(tK + ch * 32, dk);
-            tmem_ld32(tV + ch * 32, dv);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              float ex = fmaf(dk[i], scale, nb);
-              if constexpr (kCenter) ex -= shift[r * kTile + ch * 32 + i] * scale;
-              const float val = fast_exp2(ex) * dv[i];
-              g[ch * 32 + i] = (ch < q || i < lane) ? val : 0.f;   // strictly earlier tokens only
-            }
-          }
-        }
-        tc_fence_before();
-        mbar_arrive(tmem_empty + buf);                     // TMEM buffer is free while we walk
+      if ((tile_it & 1) != wg) {
+        // the other warpgroup owns the diagonal tile: hand over this group's partial sums
+        xacc[(r & 1) * kTile + row] = acc;
+        mbar_arrive(xacc_full + (r & 1));
         ++tile_it;
-        float S = acc;
+        continue;
+      }
+      // ---- diagonal tile: Ghat of this row against the panel's earlier tokens, then the walk
+      const float u = walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, j);
+      const float thr = cw * (1.0f - 2.0f * u);
+      if (!(ok = wait_bar(tmem_full + wg, (uint32_t)(my_tiles & 1), abort_flag))) break;
+      tc_fence_after();
+      float own[32], prev[32];        // Ghat/inv_rv2 towards this warp's own 32 tokens / the 32 before them
+      {
+        float dk[32], dv[32];
+        tmem_ld32(tbase + q * 32, dk);
+        tmem_ld32(tbase + 128 + q * 32, dv);
+        tmem_ld_wait();
 #pragma unroll
-        for (int gi = 0; gi < 3; ++gi) {
-          if (gi < q) {                                    // warp-uniform
-            if (!(ok = wait_progress(progress, 4 * r + gi + 1, abort_flag))) break;
-            const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + gi * 32);
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        for (int i = 0; i < 32; ++i) {
+          float ex = fmaf(dk[i], scale, nb);
+          if constexpr (kCenter) ex -= shift[r * kTile + q * 32 + i] * scale;
+          own[i] = i < lane ? fast_exp2(ex) * dv[i] * inv_rv2 : 0.f;       // strictly earlier tokens only
+        }
+      }
+      if (q > 0) {
+        float dk[32], dv[32];
+        tmem_ld32(tbase + (q - 1) * 32, dk);
+        tmem_ld32(tbase + 128 + (q - 1) * 32, dv);
+        tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
-              const float4 e = e4[x];
-              s0 = fmaf(g[gi * 32 + 4 * x + 0], e.x, s0);
-              s1 = fmaf(g[gi * 32 + 4 * x + 1], e.y, s1);
-              s2 = fmaf(g[gi * 32 + 4 * x + 2], e.z, s2);
-              s3 = fmaf(g[gi * 32 + 4 * x + 3], e.w, s3);
-            }
-            S += (s0 + s1) + (s2 + s3);
+        for (int i = 0; i < 32; ++i) {
+          float ex = fmaf(dk[i], scale, nb);
+          if constexpr (kCenter) ex -= shift[r * kTile + (q - 1) * 32 + i] * scale;
+          prev[i] = fast_exp2(ex) * dv[i];
+        }
+      }
+      // groups two or more before this one: their signs are (almost always) final already
+      for (int ch = 0; ch + 1 < q && ok; ++ch) {
+        if (!(ok = wait_progress(progress, 4 * r + ch + 1, abort_flag))) break;
+        float dk[32], dv[32];
+        tmem_ld32(tbase + ch * 32, dk);
+        tmem_ld32(tbase + 128 + ch * 32, dv);
+        tmem_ld_wait();
+        const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + ch * 32);
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          const float4 e = e4[x];
+          const float ev[4] = {e.x, e.y, e.z, e.w};
+#pragma unroll
+          for (int y = 0; y < 4; ++y) {
+            const int i = 4 * x + y;
+            float ex = fmaf(dk[i], scale, nb);
+            if constexpr (kCenter) ex -= shift[r * kTile + ch * 32 + i] * scale;
+            acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
           }
         }
-        if (!ok) break;
-        // the sequential walk over this warp's 32 tokens
-        float own[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          own[i] = 0.f;
-#pragma unroll
-          for (int qq = 0; qq < 4; ++qq)
-            if (qq == q) own[i] = g[qq * 32 + i];          // warp-uniform select of the own block
-        }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float dec = S < thr ? inv_rv2 : -inv_rv2;
-          const float ei = __shfl_sync(0xffffffffu, dec, i);
-          S = fmaf(ei, own[i], S);                         // own[i] = 0 once this lane's token is decided
-        }
-        const bool plus = S < thr;
-        etas[j] = plus ? inv_rv2 : -inv_rv2;
-        eta8[j] = plus ? 1 : -1;
-        if (fabsf(S) > cw) ++fails;                        // FAIL of Algorithm 2: counted; the decision is the clamped one
-        if (C.dbg_off >= 0) {
-          dbg_S[C.dbg_off + j] = S;
-          dbg_p[C.dbg_off + j] = 0.5f - fminf(fmaxf(S, -cw), cw) / (2.0f * cw);
-        }
-        __syncwarp();
-        if (lane == 0) st_release(progress, 4 * r + q + 1);
       }
+      tc_fence_before();
+      mbar_arrive(tmem_empty + wg);                      // the TMEM buffer is free while we walk
+      ++my_tiles;
+      ++tile_it;
+      if (!ok) break;
+      // partial sums of the tiles the other warpgroup drained for this panel
+      if (!(ok = wait_bar(xacc_full + (r & 1), (uint32_t)((r >> 1) & 1), abort_flag))) break;
+      float S_pre = acc + xacc[(r & 1) * kTile + row];
+      if (q > 0) {
+        if (!(ok = wait_progress(progress, 4 * r + q, abort_flag))) break;     // the 32 tokens just before
+        const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + (q - 1) * 32);
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          const float4 e = e4[x];
+          s0 = fmaf(prev[4 * x + 0], e.x, s0);
+          s1 = fmaf(prev[4 * x + 1], e.y, s1);
+          s2 = fmaf(prev[4 * x + 2], e.z, s2);
+          s3 = fmaf(prev[4 * x + 3], e.w, s3);
+        }
+        S_pre += (s0 + s1) + (s2 + s3);
+      }
+      // The walk over this warp's 32 tokens.  eta_l depends only on eta_{<l}, so the sequential
+      // solution is the unique fixed point of "decide every token from the current signs"; each
+      // sweep makes at least one more leading token final, and a sweep that changes nothing
+      // proves the fixed point.  With small Ghat two sweeps suffice; 32 always do.
+      float S = S_pre;
+      unsigned mask = __ballot_sync(0xffffffffu, S < thr);
+#pragma unroll 1
+      for (int sweep = 0; sweep < 33; ++sweep) {
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          s0 += (mask >> (i + 0)) & 1u ? own[i + 0] : -own[i + 0];
+          s1 += (mask >> (i + 1)) & 1u ? own[i + 1] : -own[i + 1];
+          s2 += (mask >> (i + 2)) & 1u ? own[i + 2] : -own[i + 2];
+          s3 += (mask >> (i + 3)) & 1u ? own[i + 3] : -own[i + 3];
+        }
+        S = S_pre + ((s0 + s1) + (s2 + s3));
+        const unsigned next = __ballot_sync(0xffffffffu, S < thr);
+        if (next == mask) break;
+        mask = next;
+      }
+      const bool plus = (mask >> lane) & 1u;
+      etas[j] = plus ? inv_rv2 : -inv_rv2;
+      eta8[j] = plus ? 1 : -1;
+      if (fabsf(S) > cw) ++fails;                          // FAIL of Algorithm 2: counted; the decision is the clamped one
+      if (C.dbg_off >= 0) {
+        dbg_S[C.dbg_off + j] = S;
+        dbg_p[C.dbg_off + j] = 0.5f - fminf(fmaxf(S, -cw), cw) / (2.0f * cw);
+      }
+      __syncwarp();
+      if (lane == 0) st_release(progress, 4 * r + q + 1);
     }
     fails = (int)__reduce_add_sync(0xffffffffu, (unsigned)fails);
     if (lane == 0 && fails) atomicAdd(fail_count, (unsigned long long)fails);
@@ -397,12 +447,12 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       if (C.dbg_off >= 0) dbg_eta[C.dbg_off + i] = e;
     }
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 128; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 160; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
