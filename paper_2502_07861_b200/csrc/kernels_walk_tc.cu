@@ -3,10 +3,10 @@
 // One CTA per call.  The call's t x t kernel matrix
 //   Ghat_ij = exp((<k_i,k_j> - r_key^2)/sqrt d) <v_i,v_j> / r_value^2      (proof of Theorem 3.2)
 // is visited in 128 x 128 tiles of its lower triangle, row panel by row panel.  For a tile,
-// TMA brings the bf16 rows of K and V into 128B-swizzled shared memory, one thread issues
-// tcgen05.mma (bf16 x bf16 -> fp32) for K_r K_c^T and V_r V_c^T into two TMEM accumulators,
-// and two epilogue warpgroups (thread = row, alternating tiles) read them back with tcgen05.ld,
-// apply exp2/scale/product and fold the tile into the row's running correlation
+// TMA brings the bf16 rows of K and V into 128B-swizzled shared memory, tcgen05.mma
+// (bf16 x bf16 -> fp32) forms K_r K_c^T and V_r V_c^T in two TMEM accumulators, and two
+// epilogue warpgroups (thread = row, 64 columns of the tile each) read them back with
+// tcgen05.ld, apply exp2/scale/product and fold the tile into the row's running correlation
 //   S_j = sum_{i<j} eta_i Ghat_ij
 // with the signs of earlier panels.  The diagonal tile feeds the walk: warp q owns rows
 // 32q..32q+31 of the panel, lane l owns one token,
@@ -14,9 +14,8 @@
 // u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).  Inside a 32-token
 // group the sequential recurrence is solved by sweeps (decide all tokens from the current
 // signs, repeat until nothing changes), which reaches exactly the sequential result.
-// TMEM is double buffered (2 x 256 columns, one buffer per warpgroup), so the tensor core
-// works on the next tile while an epilogue drains the previous one; Ghat never touches
-// global memory.
+// TMEM is double buffered (2 x 256 columns); an epilogue hands its buffer back as soon as the
+// accumulator values are in registers.  Ghat never touches global memory.
 //
 // Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
 // roles leave their loops, TMEM is freed and the kernel returns.
@@ -97,24 +96,38 @@ __device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled bf16 operand: rows of 128 bytes,
 // 8-row groups 1024 bytes apart (stride byte offset), version 1, layout type SWIZZLE_128B.
-__device__ inline uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                  // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset
-  d |= (uint64_t)1 << 46;                  // descriptor version
-  d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
-  return d;
-}
+// Only the low word depends on the address: (addr >> 4) in bits [0,14), leading byte offset 1
+// (unused for swizzled K-major) in bits [16,30).  Stepping 16 elements along K adds 32 bytes,
+// i.e. 2 to the low word; the second 64-column half of a tile sits kHalfBytes further.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ inline uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
 // kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = N = 128.
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
-__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+// A tcgen05.mma is issued at the rate the tensor core retires them, so every other instruction
+// of the issuing thread is idle time of the pipe: descriptors come as ready-made words and the
+// accumulate flag is a compile-time constant.
+template <int kAccumulate>
+__device__ inline void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate) : "memory");
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "n"(kAccumulate), "r"(kInstrDesc) : "memory");
+}
+// The 8 K-steps of one 128 x 128 x 128 product: A and B tiles given by their descriptor low words.
+__device__ inline void umma_tile(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
+  constexpr uint32_t kHalf = kHalfBytes >> 4;
+  umma_bf16<0>(d_tmem, a_lo, b_lo);
+  umma_bf16<1>(d_tmem, a_lo + 2, b_lo + 2);
+  umma_bf16<1>(d_tmem, a_lo + 4, b_lo + 4);
+  umma_bf16<1>(d_tmem, a_lo + 6, b_lo + 6);
+  umma_bf16<1>(d_tmem, a_lo + kHalf, b_lo + kHalf);
+  umma_bf16<1>(d_tmem, a_lo + kHalf + 2, b_lo + kHalf + 2);
+  umma_bf16<1>(d_tmem, a_lo + kHalf + 4, b_lo + kHalf + 4);
+  umma_bf16<1>(d_tmem, a_lo + kHalf + 6, b_lo + kHalf + 6);
 }
 __device__ inline void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -171,8 +184,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   uint64_t* col_empty = bars + 4;    // [2]
   uint64_t* tmem_full = bars + 6;    // [2]
   uint64_t* tmem_empty = bars + 8;   // [2]
-  uint64_t* xacc_full = bars + 10;   // [2]
-  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 12);
+  uint64_t* xacc_full = bars + 10;   // [2][4]: per panel parity and warp quarter
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 18);
   int* progress = reinterpret_cast<int*>(tmem_ptr_s + 1);
   int* abort_flag = progress + 1;
 
@@ -184,9 +197,9 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     mbar_init(row_full, 1); mbar_init(row_empty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(col_full + i, 1); mbar_init(col_empty + i, 1);
-      mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 128);
-      mbar_init(xacc_full + i, 128);
+      mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 256);
     }
+    for (int i = 0; i < 8; ++i) mbar_init(xacc_full + i, 32);
     *progress = 0; *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -232,31 +245,24 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     if (lane == 0) {
       int tile_it = 0, col_it = 0;
       bool ok = true;
-      const uint32_t kr = smem_u32(sm + Smem::kKr), vr = smem_u32(sm + Smem::kVr);
+      const uint32_t kr = umma_desc_lo(smem_u32(sm + Smem::kKr)), vr = umma_desc_lo(smem_u32(sm + Smem::kVr));
+      const uint32_t st0 = umma_desc_lo(smem_u32(sm + Smem::kStage0));
       for (int r = 0; r < P && ok; ++r) {
         if (!(ok = wait_bar(row_full, (uint32_t)(r & 1), abort_flag))) break;
         for (int c = 0; c <= r; ++c, ++tile_it) {
-          const int buf = tile_it & 1;                 // tile i belongs to epilogue warpgroup i & 1
+          const int buf = tile_it & 1;
           if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((tile_it >> 1) & 1) ^ 1), abort_flag))) break;
           uint32_t kb = kr, vb = vr;
           const int s = col_it & 1;
           if (c < r) {
             if (!(ok = wait_bar(col_full + s, (uint32_t)((col_it >> 1) & 1), abort_flag))) break;
-            kb = smem_u32(sm + Smem::kStage0 + (uint32_t)s * 2 * kTileBytes);
-            vb = kb + kTileBytes;
+            kb = st0 + (uint32_t)s * ((2 * kTileBytes) >> 4);
+            vb = kb + (kTileBytes >> 4);
           }
           tc_fence_after();
-          const uint32_t dK = tmem_base + (uint32_t)buf * 256u, dV = dK + 128u;
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-            umma_bf16(dK, umma_desc(kr + off), umma_desc(kb + off), kk > 0);
-          }
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-            umma_bf16(dV, umma_desc(vr + off), umma_desc(vb + off), kk > 0);
-          }
+          const uint32_t dK = tmem_base + (uint32_t)buf * 256u;
+          umma_tile(dK, kr, kb);
+          umma_tile(dK + 128u, vr, vb);
           if (c < r) { umma_commit(col_empty + s); ++col_it; }
           else umma_commit(row_empty);
           umma_commit(tmem_full + buf);
@@ -266,9 +272,10 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ two epilogue warpgroups
-    // Tiles are numbered in issue order; warpgroup wg drains tiles i with (i & 1) == wg from
-    // TMEM buffer wg.  Both keep a partial running correlation per row of the current panel;
-    // the group that gets the diagonal tile collects the other's partial and walks the panel.
+    // Every tile is drained by both warpgroups: group wg takes columns 64 wg .. 64 wg + 63 of the
+    // tile (thread = row).  Each thread keeps a partial running correlation of its row; at the
+    // diagonal tile the panel's owner group (alternating) collects the other group's partial and
+    // walks the panel, while the other group folds in the diagonal tile's older columns.
     const int wg = warp >> 2;
     const int q = warp & 3;                   // quarter of the panel = TMEM lane quadrant
     const int row = 32 * q + lane;
@@ -280,62 +287,89 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
     const float scale = 1.4426950408889634f * G.inv_sqrt_d;
     const float cw = G.c;
-    const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)wg * 256u;
+    const uint32_t tlane = tmem_base + ((uint32_t)(32 * q) << 16);
     const float* shift = kCenter ? tok_shift + (size_t)call * t : nullptr;
-    int tile_it = 0, my_tiles = 0, fails = 0;
+    int tile_it = 0, fails = 0;
     bool ok = true;
+
+    // acc += sum over 32 columns of Ghat' * sign, from accumulator values already in registers
+    auto fold_regs = [&](const float (&dk)[32], const float (&dv)[32], const float* signs, int shift_base, float nb,
+                         float acc) -> float {
+      const float4* e4 = reinterpret_cast<const float4*>(signs);
+#pragma unroll
+      for (int x = 0; x < 8; ++x) {
+        const float4 e = e4[x];
+        const float ev[4] = {e.x, e.y, e.z, e.w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+          const int i = 4 * x + y;
+          float ex = fmaf(dk[i], scale, nb);
+          if constexpr (kCenter) ex -= shift[shift_base + i] * scale;
+          acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
+        }
+      }
+      return acc;
+    };
+    auto fold_chunk = [&](uint32_t tb, int ch, const float* signs, int shift_base, float nb, float acc) -> float {
+      float dk[32], dv[32];
+      tmem_ld32(tb + ch * 32, dk);
+      tmem_ld32(tb + 128 + ch * 32, dv);
+      tmem_ld_wait();
+      return fold_regs(dk, dv, signs + ch * 32, shift_base + ch * 32, nb, acc);
+    };
+
     for (int r = 0; r < P && ok; ++r) {
       const int j = r * kTile + row;                      // this thread's token in the panel
       float nb = -rk2 * scale;                            // exponent offset of this row
       if constexpr (kCenter) nb -= shift[j] * scale;
       float acc = 0.f;
       for (int c = 0; c < r && ok; ++c, ++tile_it) {
-        if ((tile_it & 1) != wg) continue;
+        const int buf = tile_it & 1;
         if (!(ok = wait_progress(progress, 4 * c + 4, abort_flag))) break;     // signs of panel c are final
-        if (!(ok = wait_bar(tmem_full + wg, (uint32_t)(my_tiles & 1), abort_flag))) break;
+        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
         tc_fence_after();
-#pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          float dk[32], dv[32];
-          tmem_ld32(tbase + ch * 32, dk);
-          tmem_ld32(tbase + 128 + ch * 32, dv);
-          tmem_ld_wait();
-          const float4* e4 = reinterpret_cast<const float4*>(etas + c * kTile + ch * 32);
-#pragma unroll
-          for (int x = 0; x < 8; ++x) {
-            const float4 e = e4[x];
-            const float ev[4] = {e.x, e.y, e.z, e.w};
-#pragma unroll
-            for (int y = 0; y < 4; ++y) {
-              const int i = 4 * x + y;
-              float ex = fmaf(dk[i], scale, nb);
-              if constexpr (kCenter) ex -= shift[c * kTile + ch * 32 + i] * scale;
-              acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
-            }
-          }
-        }
+        const uint32_t tb = tlane + (uint32_t)buf * 256u;
+        // pull this group's 64 columns of both accumulators into registers and hand the TMEM
+        // buffer back at once; the arithmetic then overlaps the next tiles' MMAs
+        float dk0[32], dv0[32], dk1[32], dv1[32];
+        tmem_ld32(tb + (2 * wg) * 32, dk0);
+        tmem_ld32(tb + 128 + (2 * wg) * 32, dv0);
+        tmem_ld32(tb + (2 * wg + 1) * 32, dk1);
+        tmem_ld32(tb + 128 + (2 * wg + 1) * 32, dv1);
+        tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(tmem_empty + wg);
-        ++my_tiles;
+        mbar_arrive(tmem_empty + buf);
+        acc = fold_regs(dk0, dv0, etas + c * kTile + (2 * wg) * 32, c * kTile + (2 * wg) * 32, nb, acc);
+        acc = fold_regs(dk1, dv1, etas + c * kTile + (2 * wg + 1) * 32, c * kTile + (2 * wg + 1) * 32, nb, acc);
       }
       if (!ok) break;
-      if ((tile_it & 1) != wg) {
-        // the other warpgroup owns the diagonal tile: hand over this group's partial sums
+      // ---- diagonal tile
+      const int buf = tile_it & 1;
+      if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+      tc_fence_after();
+      const uint32_t tb = tlane + (uint32_t)buf * 256u;
+      ++tile_it;
+      if (wg != (r & 1)) {
+        // helper group: columns of the groups two or more before this warp's, then hand over
+        for (int ch = 0; ch + 1 < q && ok; ++ch) {
+          if (!(ok = wait_progress(progress, 4 * r + ch + 1, abort_flag))) break;
+          acc = fold_chunk(tb, ch, etas + r * kTile, r * kTile, nb, acc);
+        }
+        tc_fence_before();
+        mbar_arrive(tmem_empty + buf);
+        if (!ok) break;
         xacc[(r & 1) * kTile + row] = acc;
-        mbar_arrive(xacc_full + (r & 1));
-        ++tile_it;
+        mbar_arrive(xacc_full + (r & 1) * 4 + q);
         continue;
       }
-      // ---- diagonal tile: Ghat of this row against the panel's earlier tokens, then the walk
+      // owner group: Ghat of this row against its warp's own 32 tokens and the 32 before them
       const float u = walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, j);
       const float thr = cw * (1.0f - 2.0f * u);
-      if (!(ok = wait_bar(tmem_full + wg, (uint32_t)(my_tiles & 1), abort_flag))) break;
-      tc_fence_after();
-      float own[32], prev[32];        // Ghat/inv_rv2 towards this warp's own 32 tokens / the 32 before them
+      float own[32], prev[32];
       {
         float dk[32], dv[32];
-        tmem_ld32(tbase + q * 32, dk);
-        tmem_ld32(tbase + 128 + q * 32, dv);
+        tmem_ld32(tb + q * 32, dk);
+        tmem_ld32(tb + 128 + q * 32, dv);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -346,8 +380,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       }
       if (q > 0) {
         float dk[32], dv[32];
-        tmem_ld32(tbase + (q - 1) * 32, dk);
-        tmem_ld32(tbase + 128 + (q - 1) * 32, dv);
+        tmem_ld32(tb + (q - 1) * 32, dk);
+        tmem_ld32(tb + 128 + (q - 1) * 32, dv);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -356,34 +390,10 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
           prev[i] = fast_exp2(ex) * dv[i];
         }
       }
-      // groups two or more before this one: their signs are (almost always) final already
-      for (int ch = 0; ch + 1 < q && ok; ++ch) {
-        if (!(ok = wait_progress(progress, 4 * r + ch + 1, abort_flag))) break;
-        float dk[32], dv[32];
-        tmem_ld32(tbase + ch * 32, dk);
-        tmem_ld32(tbase + 128 + ch * 32, dv);
-        tmem_ld_wait();
-        const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + ch * 32);
-#pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          const float4 e = e4[x];
-          const float ev[4] = {e.x, e.y, e.z, e.w};
-#pragma unroll
-          for (int y = 0; y < 4; ++y) {
-            const int i = 4 * x + y;
-            float ex = fmaf(dk[i], scale, nb);
-            if constexpr (kCenter) ex -= shift[r * kTile + ch * 32 + i] * scale;
-            acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
-          }
-        }
-      }
       tc_fence_before();
-      mbar_arrive(tmem_empty + wg);                      // the TMEM buffer is free while we walk
-      ++my_tiles;
-      ++tile_it;
-      if (!ok) break;
-      // partial sums of the tiles the other warpgroup drained for this panel
-      if (!(ok = wait_bar(xacc_full + (r & 1), (uint32_t)((r >> 1) & 1), abort_flag))) break;
+      mbar_arrive(tmem_empty + buf);                     // the TMEM buffer is free while we walk
+      // the other group's partial sums for this row
+      if (!(ok = wait_bar(xacc_full + (r & 1) * 4 + q, (uint32_t)((r >> 1) & 1), abort_flag))) break;
       float S_pre = acc + xacc[(r & 1) * kTile + row];
       if (q > 0) {
         if (!(ok = wait_progress(progress, 4 * r + q, abort_flag))) break;     // the 32 tokens just before
@@ -452,7 +462,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 160; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 224; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
