@@ -15,7 +15,9 @@
 // group the sequential recurrence is solved by sweeps (decide all tokens from the current
 // signs, repeat until nothing changes), which reaches exactly the sequential result.
 // TMEM is double buffered (2 x 256 columns); an epilogue hands its buffer back as soon as the
-// accumulator values are in registers.  Ghat never touches global memory.
+// accumulator values are in registers.  Each of the two products of a tile has its own issuing
+// thread and its own barriers, so that one product's waits and commits overlap the other's
+// MMAs.  Ghat never touches global memory.
 //
 // Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
 // roles leave their loops, TMEM is freed and the kernel returns.
@@ -28,8 +30,8 @@ namespace bkv {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kThreads = 320;              // warps 0-3, 4-7: two epilogue + walk warpgroups, warp 8: TMA, warp 9: MMA
-constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 352;              // warps 0-3, 4-7: two epilogue + walk warpgroups, 8: TMA, 9: MMA (K K^T), 10: MMA (V V^T)
+constexpr int kTmaWarp = 8, kMmaWarp = 9, kMmaWarpV = 10;
 constexpr uint32_t kHalfBytes = 16384;     // [128 rows][64 bf16] = one swizzle-atom column of a tile
 constexpr uint32_t kTileBytes = 32768;     // [128 rows][128 bf16]
 constexpr uint32_t kTmemCols = 512;
@@ -178,14 +180,15 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   float* xacc = etas + t;                                                 // [2][128] partial correlations handed over
   int8_t* eta8 = reinterpret_cast<int8_t*>(xacc + 2 * kTile);             // [t] signs
   uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
-  uint64_t* row_full = bars + 0;
-  uint64_t* row_empty = bars + 1;
-  uint64_t* col_full = bars + 2;     // [2]
-  uint64_t* col_empty = bars + 4;    // [2]
-  uint64_t* tmem_full = bars + 6;    // [2]
-  uint64_t* tmem_empty = bars + 8;   // [2]
-  uint64_t* xacc_full = bars + 10;   // [2][4]: per panel parity and warp quarter
-  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 18);
+  // x = 0: the K K^T product, x = 1: the V V^T product
+  uint64_t* row_full = bars + 0;     // row panel landed
+  uint64_t* xfull = bars + 1;        // [x][2] column tile of product x landed in stage s
+  uint64_t* xdone = bars + 5;        // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
+  uint64_t* xcempty = bars + 9;      // [x][2] product x no longer reads column stage s -> producer
+  uint64_t* xrempty = bars + 13;     // [x]    product x no longer reads the row panel -> producer
+  uint64_t* tmem_empty = bars + 15;  // [2] both warpgroups have drained buffer b
+  uint64_t* xacc_full = bars + 17;   // [2][4]: per panel parity and warp quarter
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 25);
   int* progress = reinterpret_cast<int*>(tmem_ptr_s + 1);
   int* abort_flag = progress + 1;
 
@@ -194,11 +197,9 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
-    mbar_init(row_full, 1); mbar_init(row_empty, 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(col_full + i, 1); mbar_init(col_empty + i, 1);
-      mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 256);
-    }
+    mbar_init(row_full, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(xfull + i, 1); mbar_init(xdone + i, 1); mbar_init(xcempty + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(xrempty + i, 1); mbar_init(tmem_empty + i, 256); }
     for (int i = 0; i < 8; ++i) mbar_init(xacc_full + i, 32);
     *progress = 0; *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -213,59 +214,70 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
 
+  // Tiles are numbered in issue order i = 0, 1, ...: panel r contributes (r,0) .. (r,r).  Tile i
+  // uses TMEM buffer i & 1 and, unless it is a diagonal tile, column stage i & 1.  Every barrier
+  // is waited on phase by phase by its one kind of waiter, and each next phase depends on that
+  // waiter having passed, so a parity wait can never be a phase behind.
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int col_it = 0;
+      int i = 0, use0 = 0, use1 = 0;      // tiles so far; column tiles that used stage 0 / 1
       bool ok = true;
       for (int r = 0; r < P && ok; ++r) {
-        if (!(ok = wait_bar(row_empty, (uint32_t)((r & 1) ^ 1), abort_flag))) break;
+        if (r > 0) {   // both products have finished the previous panel's diagonal tile
+          if (!(ok = wait_bar(xrempty + 0, (uint32_t)((r - 1) & 1), abort_flag))) break;
+          if (!(ok = wait_bar(xrempty + 1, (uint32_t)((r - 1) & 1), abort_flag))) break;
+        }
         const int y = (int)(C.src_row + (int64_t)r * kTile);
         mbar_expect_tx(row_full, 2 * kTileBytes);
         tma_load_2d(sm + Smem::kKr, &tmK, 0, y, row_full);
         tma_load_2d(sm + Smem::kKr + kHalfBytes, &tmK, 64, y, row_full);
         tma_load_2d(sm + Smem::kVr, &tmV, 0, y, row_full);
         tma_load_2d(sm + Smem::kVr + kHalfBytes, &tmV, 64, y, row_full);
-        for (int c = 0; c < r; ++c, ++col_it) {
-          const int s = col_it & 1;
-          if (!(ok = wait_bar(col_empty + s, (uint32_t)(((col_it >> 1) & 1) ^ 1), abort_flag))) break;
+        for (int c = 0; c < r; ++c, ++i) {
+          const int s = i & 1;
+          const int n = s ? use1 : use0;                              // earlier users of this stage
+          if (s) ++use1; else ++use0;
           unsigned char* st = sm + Smem::kStage0 + (uint32_t)s * 2 * kTileBytes;
           const int yc = (int)(C.src_row + (int64_t)c * kTile);
-          mbar_expect_tx(col_full + s, 2 * kTileBytes);
-          tma_load_2d(st, &tmK, 0, yc, col_full + s);
-          tma_load_2d(st + kHalfBytes, &tmK, 64, yc, col_full + s);
-          tma_load_2d(st + kTileBytes, &tmV, 0, yc, col_full + s);
-          tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, yc, col_full + s);
+          if (n > 0 && !(ok = wait_bar(xcempty + s, (uint32_t)((n - 1) & 1), abort_flag))) break;
+          mbar_expect_tx(xfull + s, kTileBytes);
+          tma_load_2d(st, &tmK, 0, yc, xfull + s);
+          tma_load_2d(st + kHalfBytes, &tmK, 64, yc, xfull + s);
+          if (n > 0 && !(ok = wait_bar(xcempty + 2 + s, (uint32_t)((n - 1) & 1), abort_flag))) break;
+          mbar_expect_tx(xfull + 2 + s, kTileBytes);
+          tma_load_2d(st + kTileBytes, &tmV, 0, yc, xfull + 2 + s);
+          tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, yc, xfull + 2 + s);
         }
+        ++i;   // the diagonal tile loads nothing
       }
     }
     __syncwarp();
-  } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == kMmaWarp || warp == kMmaWarpV) {
+    // ------------------------------------------------------------------ MMA issuers (K K^T and V V^T)
     if (lane == 0) {
-      int tile_it = 0, col_it = 0;
+      const int x = warp == kMmaWarpV ? 1 : 0;
+      int i = 0, use0 = 0, use1 = 0;
       bool ok = true;
-      const uint32_t kr = umma_desc_lo(smem_u32(sm + Smem::kKr)), vr = umma_desc_lo(smem_u32(sm + Smem::kVr));
-      const uint32_t st0 = umma_desc_lo(smem_u32(sm + Smem::kStage0));
+      const uint32_t arow = umma_desc_lo(smem_u32(sm + (x ? Smem::kVr : Smem::kKr)));
+      const uint32_t st0 = umma_desc_lo(smem_u32(sm + Smem::kStage0 + (x ? kTileBytes : 0u)));
       for (int r = 0; r < P && ok; ++r) {
         if (!(ok = wait_bar(row_full, (uint32_t)(r & 1), abort_flag))) break;
-        for (int c = 0; c <= r; ++c, ++tile_it) {
-          const int buf = tile_it & 1;
-          if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((tile_it >> 1) & 1) ^ 1), abort_flag))) break;
-          uint32_t kb = kr, vb = vr;
-          const int s = col_it & 1;
+        for (int c = 0; c <= r; ++c, ++i) {
+          const int buf = i & 1;
+          if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag))) break;
+          uint32_t b = arow;
           if (c < r) {
-            if (!(ok = wait_bar(col_full + s, (uint32_t)((col_it >> 1) & 1), abort_flag))) break;
-            kb = st0 + (uint32_t)s * ((2 * kTileBytes) >> 4);
-            vb = kb + (kTileBytes >> 4);
+            const int n = buf ? use1 : use0;
+            if (buf) ++use1; else ++use0;
+            if (!(ok = wait_bar(xfull + 2 * x + buf, (uint32_t)(n & 1), abort_flag))) break;
+            b = st0 + (uint32_t)buf * ((2 * kTileBytes) >> 4);
           }
           tc_fence_after();
-          const uint32_t dK = tmem_base + (uint32_t)buf * 256u;
-          umma_tile(dK, kr, kb);
-          umma_tile(dK + 128u, vr, vb);
-          if (c < r) { umma_commit(col_empty + s); ++col_it; }
-          else umma_commit(row_empty);
-          umma_commit(tmem_full + buf);
+          umma_tile(tmem_base + (uint32_t)buf * 256u + (x ? 128u : 0u), arow, b);
+          if (c < r) umma_commit(xcempty + 2 * x + buf);
+          else umma_commit(xrempty + x);
+          umma_commit(xdone + 2 * x + buf);
         }
       }
     }
@@ -326,7 +338,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       for (int c = 0; c < r && ok; ++c, ++tile_it) {
         const int buf = tile_it & 1;
         if (!(ok = wait_progress(progress, 4 * c + 4, abort_flag))) break;     // signs of panel c are final
-        if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+        if (!(ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+        if (!(ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
         tc_fence_after();
         const uint32_t tb = tlane + (uint32_t)buf * 256u;
         // pull this group's 64 columns of both accumulators into registers and hand the TMEM
@@ -345,7 +358,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       if (!ok) break;
       // ---- diagonal tile
       const int buf = tile_it & 1;
-      if (!(ok = wait_bar(tmem_full + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+      if (!(ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
+      if (!(ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
       tc_fence_after();
       const uint32_t tb = tlane + (uint32_t)buf * 256u;
       ++tile_it;
@@ -462,7 +476,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 224; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 256; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
