@@ -160,6 +160,35 @@ __device__ inline float fast_exp2(float x) {
   return y;
 }
 
+// 2^x for a pair of values on the FMA pipe (the special-function unit delivers 16 ex2 per clock
+// and SM, which is as many cycles per tile as the tensor core needs for its MMAs; moving part of
+// the exponentials here takes the unit off the critical path).  Cody-Waite: x = n + f with n the
+// nearest integer (magic-number rounding) and f in [-1/2, 1/2]; 2^f by a degree-5 polynomial
+// (coefficients from a Remez fit of 2^f on [-1/2, 1/2], relative error 7.5e-8; 2.3e-7 when
+// evaluated in fp32); 2^n by adding n to the exponent field.  Valid for x in [-126, 126];
+// smaller x are clamped (result ~1e-38 instead of 0).
+__device__ inline float2 poly_exp2x2(float2 x) {
+  const float kMagic = 12582912.0f;   // 1.5 * 2^23
+  x.x = fmaxf(x.x, -126.0f);
+  x.y = fmaxf(x.y, -126.0f);
+  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), x);
+  float2 p = make_float2(0x1.5c08e6p-10f, 0x1.5c08e6p-10f);
+  p = __ffma2_rn(p, f, make_float2(0x1.3d0c52p-7f, 0x1.3d0c52p-7f));
+  p = __ffma2_rn(p, f, make_float2(0x1.c6b6e4p-5f, 0x1.c6b6e4p-5f));
+  p = __ffma2_rn(p, f, make_float2(0x1.ebf918p-3f, 0x1.ebf918p-3f));
+  p = __ffma2_rn(p, f, make_float2(0x1.62e428p-1f, 0x1.62e428p-1f));
+  p = __ffma2_rn(p, f, make_float2(0x1.000002p+0f, 0x1.000002p+0f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return r;
+}
+// Of the 16 column pairs of a 32-column chunk, pairs with (index % 8) < kPolyOf8 take the
+// polynomial path, the others the special-function unit.
+constexpr int kPolyOf8 = 3;
+
 struct Smem {
   // operand tiles first (1024-byte aligned for the 128B swizzle)
   static constexpr uint32_t kKr = 0, kVr = kTileBytes, kStage0 = 2 * kTileBytes;   // stage: K then V
@@ -304,23 +333,43 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     int tile_it = 0, fails = 0;
     bool ok = true;
 
-    // acc += sum over 32 columns of Ghat' * sign, from accumulator values already in registers
+    // acc += sum over 32 columns of Ghat' * sign, from accumulator values already in registers;
+    // two columns at a time with packed fp32 instructions
     auto fold_regs = [&](const float (&dk)[32], const float (&dv)[32], const float* signs, int shift_base, float nb,
                          float acc) -> float {
       const float4* e4 = reinterpret_cast<const float4*>(signs);
+      if constexpr (kCenter) {
 #pragma unroll
-      for (int x = 0; x < 8; ++x) {
-        const float4 e = e4[x];
-        const float ev[4] = {e.x, e.y, e.z, e.w};
+        for (int x = 0; x < 8; ++x) {
+          const float4 e = e4[x];
+          const float ev[4] = {e.x, e.y, e.z, e.w};
 #pragma unroll
-        for (int y = 0; y < 4; ++y) {
-          const int i = 4 * x + y;
-          float ex = fmaf(dk[i], scale, nb);
-          if constexpr (kCenter) ex -= shift[shift_base + i] * scale;
-          acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
+          for (int y = 0; y < 4; ++y) {
+            const int i = 4 * x + y;
+            const float ex = fmaf(dk[i], scale, nb) - shift[shift_base + i] * scale;
+            acc = fmaf(fast_exp2(ex) * dv[i], ev[y], acc);
+          }
         }
+        return acc;
+      } else {
+        float2 acc2 = make_float2(acc, 0.f);
+        const float2 sc2 = make_float2(scale, scale), nb2 = make_float2(nb, nb);
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          const float4 e = e4[x];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int i = 4 * x + 2 * h, pair = 2 * x + h;
+            const float2 ex = __ffma2_rn(make_float2(dk[i], dk[i + 1]), sc2, nb2);
+            float2 ee;
+            if ((pair & 7) < kPolyOf8) ee = poly_exp2x2(ex);
+            else ee = make_float2(fast_exp2(ex.x), fast_exp2(ex.y));
+            const float2 g = __fmul2_rn(ee, make_float2(dv[i], dv[i + 1]));
+            acc2 = __ffma2_rn(g, h ? make_float2(e.z, e.w) : make_float2(e.x, e.y), acc2);
+          }
+        }
+        return acc2.x + acc2.y;
       }
-      return acc;
     };
     auto fold_chunk = [&](uint32_t tb, int ch, const float* signs, int shift_base, float nb, float acc) -> float {
       float dk[32], dv[32];
