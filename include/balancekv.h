@@ -58,8 +58,9 @@ typedef struct balancekv_config {
   int32_t recent_window; /* W >= 0: the newest W tokens of a stream never enter a call        */
   int32_t center_keys;   /* 1: subtract the call's mean key inside the kernel only
                             (the stored keys are untouched); 0 (default): off                 */
-  int32_t gram_path;     /* 0 = automatic, 1 = CUDA-core (fp32 FMA) kernel, 2 = tensor-core
-                            (tcgen05) kernel; 2 needs bf16, d = 128, t multiple of 128        */
+  int32_t gram_path;     /* 0 = automatic, 1 = CUDA-core (fp32 FMA) kernels for the walk and for
+                            decode, 2 = tensor-core (tcgen05) walk kernel; 2 needs bf16,
+                            d = 128, t multiple of 128                                         */
   int32_t reserved;
   uint64_t seed;         /* Philox key; sequence s uses seed + s                              */
   float delta;           /* failure probability of Algorithm 2; <= 0 means 1/N^2              */

@@ -17,6 +17,11 @@ namespace bkv {
 bool walk_tc_supported(const Geom& G);
 cudaError_t walk_tc_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** tmaps_out);
 void walk_tc_release(void* tmaps);
+bool decode_mma_supported(const Geom& G);
+cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out);
+void decode_mma_release(void* maps);
+cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
+                              int splits, int* status, const void* maps, cudaStream_t st);
 }  // namespace bkv
 
 #define BKV_CUDA(expr)                                                                    \
@@ -51,6 +56,7 @@ struct balancekv_ctx {
   int max_splits = 1;
   bool use_tc = false;
   void* tmaps = nullptr;
+  void* decode_maps = nullptr;   // tensor maps of the tensor-core decode kernel (bf16, d = 128)
 
   // descriptor ring: two halves of pinned host memory mirrored on the device
   char* h_ring = nullptr;
@@ -260,6 +266,10 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   if ((rc = dev_alloc(c, &c->A.idx, (size_t)c->total_rows))) return fail(rc);
   if ((rc = dev_alloc(c, &c->A.seg, (size_t)c->n_streams * (T + 1)))) return fail(rc);
   if (cudaMemset(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (T + 1)) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  // rows that were never written must hold finite numbers: tiles of the decode kernels may
+  // cover rows past a segment's end, which are masked to weight zero but still multiplied
+  if (cudaMemset(c->A.K, 0, (size_t)c->total_rows * row_bytes) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  if (cudaMemset(c->A.V, 0, (size_t)c->total_rows * row_bytes) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   if (T > 0) {
     if ((rc = dev_alloc(c, &c->d_stats, (size_t)c->max_calls))) return fail(rc);
     if ((rc = dev_alloc(c, &c->d_eta, (size_t)c->max_calls * t))) return fail(rc);
@@ -281,6 +291,9 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   for (int i = 0; i < 2; ++i)
     if (cudaEventCreateWithFlags(&c->ring_ev[i], cudaEventDisableTiming) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
 
+  if (f.gram_path != 1 && decode_mma_supported(G)) {
+    if (decode_mma_prepare(G, c->A, c->total_rows, &c->decode_maps) != cudaSuccess) c->decode_maps = nullptr;
+  }
   const bool tc_ok = walk_tc_supported(G) && c->total_rows < ((int64_t)1 << 31);
   if (f.gram_path == 2 && !tc_ok) return fail(BALANCEKV_E_INVAL);
   c->use_tc = T > 0 && tc_ok && f.gram_path != 1;
@@ -302,6 +315,7 @@ int balancekv_destroy(balancekv_ctx* c) {
   if (!c) return BALANCEKV_E_INVAL;
   cudaDeviceSynchronize();
   walk_tc_release(c->tmaps);
+  decode_mma_release(c->decode_maps);
   void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
                   c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
                   c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out};
@@ -554,8 +568,12 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
   const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
   {
     ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
-    BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
-                           static_cast<cudaStream_t>(stream)));
+    if (c->decode_maps)
+      BKV_CUDA(launch_decode_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
+                                 static_cast<cudaStream_t>(stream)));
+    else
+      BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
+                             static_cast<cudaStream_t>(stream)));
   }
   c->kernels_launched++;
   return BALANCEKV_OK;

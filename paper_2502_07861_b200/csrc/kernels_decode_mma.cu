@@ -1,0 +1,365 @@
+// Split-K decode attention over the weighted compressed cache, bf16 / d = 128, on tensor cores.
+//
+//   out = sum_i w_i e^{<k_i,q>/sqrt d} v_i / sum_i w_i e^{<k_i,q>/sqrt d},   w_i = 2^level(i)
+//
+// (output ratio of Algorithm 1 / estimator of Theorem 3.3 over the sets C^T..C^0 of a stream;
+// Eq. (1) when every token sits in C^0).  The g <= 8 query heads of a KV head form the rows of a
+// 16-row MMA tile, so q.K^T and p.V each cost one mma.sync.m16n8k16 per 8 tokens x 16 dims: at
+// g = 5 the CUDA-core formulation needs ~65 instructions per token and is issue bound far below
+// HBM speed, this one needs ~6.
+//
+// Grid (streams of the layer, splits), 4 warps.  A CTA walks its share of the stream's 64-token
+// tiles through a 3-stage ring filled by TMA (tensor maps over the K and V arenas, boxes of
+// 64 dims x 64 rows, 128-byte swizzle, so ldmatrix reads are bank-conflict free).  Warp w owns
+// tokens 16w..16w+15 of a tile and keeps a private online softmax (running max, sum, 16 x 128
+// accumulator) in registers; warps merge through shared memory, splits through a global scratch
+// and a ticket counter (the last CTA of a stream combines; nobody waits).
+// Rows of a tile beyond a segment's end are masked in the scores; their V rows are whatever the
+// arena holds there (zero-initialised at creation or finite older rows) times an exact zero.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace bkv {
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kWarps = 4;
+constexpr int kStages = 3;
+constexpr int kTN = 64;                      // tokens per tile
+constexpr int kD = 128;
+constexpr uint32_t kHalf = kTN * 128;        // bytes of one [64 tokens][64 dims] bf16 box
+constexpr uint32_t kTensorBytes = 2 * kHalf; // K (or V) tile: two boxes
+constexpr uint32_t kStageBytes = 2 * kTensorBytes;
+constexpr long long kWaitCycles = 4000000000LL;
+constexpr int PS = kD + 2;                   // partial row: acc[D], max, sum
+
+struct DecodeMaps {
+  CUtensorMap k, v;
+};
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ inline void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ inline void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+  return true;
+}
+__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
+}
+__device__ inline void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ inline void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ inline void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ inline uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+// Byte offset of (token row, 16-byte chunk of dims) inside a K or V tile: two 64-dim boxes of
+// 64 rows x 128 bytes, chunk index XORed with (row % 8) by the 128-byte swizzle.
+__device__ inline uint32_t tile_off(int token, int chunk16) {   // chunk16 in [0, 16)
+  return (uint32_t)(chunk16 >> 3) * kHalf + (uint32_t)token * 128u + (uint32_t)(((chunk16 & 7) ^ (token & 7)) << 4);
+}
+
+struct TileRef {
+  int64_t row;
+  int rows, level;
+};
+__device__ inline TileRef locate_tile(int tile, const int* lvl_tiles, const Seg* seg, int T, int64_t stream_base,
+                                      const int32_t* region_off) {
+  TileRef r{0, 0, 0};
+  for (int l = T; l >= 0; --l) {
+    const int nt = lvl_tiles[l];
+    if (tile < nt) {
+      r.level = l;
+      r.row = stream_base + region_off[l] + seg[l].start + (int64_t)tile * kTN;
+      r.rows = min(kTN, seg[l].len - tile * kTN);
+      return r;
+    }
+    tile -= nt;
+  }
+  return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
+                  float* __restrict__ part, unsigned* __restrict__ tickets, int* __restrict__ status,
+                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + kStages * kStageBytes);
+  __shared__ int lvl_tiles[kMaxLevels + 1];
+  __shared__ Seg seg_s[kMaxLevels + 1];
+  __shared__ int is_last_s;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = G.g;
+  const int sl = blockIdx.x;
+  const int seq = sl / G.H, head = sl % G.H;
+  const int stream = (seq * G.L + layer) * G.H + head;
+  const int splits = gridDim.y, split = blockIdx.y;
+  const int64_t stream_base = (int64_t)stream * G.rows_per_stream;
+
+  if (tid <= G.T) {
+    const Seg s = A.seg[(size_t)stream * (G.T + 1) + tid];
+    seg_s[tid] = s;
+    lvl_tiles[tid] = (s.len + kTN - 1) / kTN;
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  int n_tiles = 0;
+  for (int l = 0; l <= G.T; ++l) n_tiles += lvl_tiles[l];
+  const int t_begin = (int)((long long)n_tiles * split / splits);
+  const int t_end = (int)((long long)n_tiles * (split + 1) / splits);
+  const int my_tiles = t_end - t_begin;
+
+  auto issue = [&](int i) {   // thread 0 only
+    const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
+    unsigned char* st = tiles + (size_t)(i % kStages) * kStageBytes;
+    uint64_t* bar = &full[i % kStages];
+    mbar_expect_tx(bar, kStageBytes);
+    tma_load_2d(st, &tmK, 0, (int)tr.row, bar);
+    tma_load_2d(st + kHalf, &tmK, 64, (int)tr.row, bar);
+    tma_load_2d(st + kTensorBytes, &tmV, 0, (int)tr.row, bar);
+    tma_load_2d(st + kTensorBytes + kHalf, &tmV, 64, (int)tr.row, bar);
+  };
+  if (tid == 0)
+    for (int i = 0; i < min(kStages, my_tiles); ++i) issue(i);
+
+  // A fragments of the query tile: row = query head of the group (rows >= g are zero)
+  const int qrow = lane >> 2, qcol = (lane & 3) * 2;
+  uint32_t qa[8][4];
+  {
+    const __nv_bfloat16* qp = q + ((size_t)seq * (G.H * g) + (size_t)head * g + qrow) * kD;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      uint32_t lo = 0, hi = 0;
+      if (qrow < g) {
+        lo = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + qcol);
+        hi = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + qcol);
+      }
+      qa[ks][0] = lo; qa[ks][1] = 0; qa[ks][2] = hi; qa[ks][3] = 0;
+    }
+  }
+  const float sc = 1.4426950408889634f * G.inv_sqrt_d;
+
+  float o[16][4];
+#pragma unroll
+  for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_run = -INFINITY, l_run = 0.f;      // of row qrow, over this thread's columns
+
+  // ldmatrix row addresses of this lane (see the fragment layouts of mma.m16n8k16)
+  const int mi = lane >> 3, mr = lane & 7;
+  const int k_tok = warp * 16 + (mi >> 1) * 8 + mr, k_chunk = mi & 1;     // K: x4 = (tok 0-7 | 8-15) x (dims lo | hi)
+  const int v_tok = warp * 16 + (mi & 1) * 8 + mr, v_chunk = mi >> 1;     // V (transposed): x4 = (dims lo | hi) x (tok 0-7 | 8-15)
+
+  bool failed = false;
+  for (int i = 0; i < my_tiles; ++i) {
+    const int s = i % kStages;
+    const bool arrived = __all_sync(0xffffffffu, mbar_wait(&full[s], (uint32_t)((i / kStages) & 1)));
+    const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
+    const uint32_t Kt = smem_u32(tiles + (size_t)s * kStageBytes), Vt = Kt + kTensorBytes;
+    if (arrived && warp * 16 < tr.rows) {
+      // ---- scores of the 16 tokens of this warp: S[16 x 16] = Q K^T
+      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        uint32_t kb[4];
+        ldsm_x4(Kt + tile_off(k_tok, ks * 2 + k_chunk), kb);
+        mma_bf16(s0, qa[ks], kb[0], kb[1]);
+        mma_bf16(s1, qa[ks], kb[2], kb[3]);
+      }
+      // this thread: row qrow, tokens tcol, tcol+1 (s0) and tcol+8, tcol+9 (s1)
+      const int tcol = warp * 16 + qcol;
+      const float lvl = (float)tr.level;
+      float x0 = tcol < tr.rows ? fmaf(s0[0], sc, lvl) : -INFINITY;
+      float x1 = tcol + 1 < tr.rows ? fmaf(s0[1], sc, lvl) : -INFINITY;
+      float x2 = tcol + 8 < tr.rows ? fmaf(s1[0], sc, lvl) : -INFINITY;
+      float x3 = tcol + 9 < tr.rows ? fmaf(s1[1], sc, lvl) : -INFINITY;
+      float mx = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run, mx);                   // finite: token 16 w of the tile is valid
+      if (__any_sync(0xffffffffu, m_new > m_run)) {
+        const float a = exp2f(m_run - m_new);                 // m_run = -inf -> 0
+        l_run *= a;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) { o[n][0] *= a; o[n][1] *= a; }
+        m_run = m_new;
+      }
+      x0 = exp2f(x0 - m_run); x1 = exp2f(x1 - m_run); x2 = exp2f(x2 - m_run); x3 = exp2f(x3 - m_run);
+      l_run += (x0 + x1) + (x2 + x3);
+      // the probabilities enter the second MMA as bf16: split them into a high and a low part
+      // (p = hi + lo to 16 bits) so that the output error stays that of the final rounding
+      const uint32_t ph[4] = {pack_bf16(x0, x1), 0u, pack_bf16(x2, x3), 0u};
+      const uint32_t pl[4] = {pack_bf16(x0 - bf16_lo(ph[0]), x1 - bf16_hi(ph[0])), 0u,
+                              pack_bf16(x2 - bf16_lo(ph[2]), x3 - bf16_hi(ph[2])), 0u};
+      // ---- O[16 x 128] += P[16 x 16] V[16 x 128]
+#pragma unroll
+      for (int nb = 0; nb < 8; ++nb) {
+        uint32_t vb[4];
+        ldsm_x4_trans(Vt + tile_off(v_tok, nb * 2 + v_chunk), vb);
+        mma_bf16(o[2 * nb], ph, vb[0], vb[1]);
+        mma_bf16(o[2 * nb], pl, vb[0], vb[1]);
+        mma_bf16(o[2 * nb + 1], ph, vb[2], vb[3]);
+        mma_bf16(o[2 * nb + 1], pl, vb[2], vb[3]);
+      }
+    }
+    // stage s fully consumed; the same barrier makes a timed-out wait a CTA-wide decision
+    if (__syncthreads_or(!arrived)) { failed = true; break; }
+    if (tid == 0 && i + kStages < my_tiles) issue(i + kStages);
+  }
+  if (failed && tid == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
+  __syncthreads();
+
+  // ---- merge the 4 warps through shared memory (the tile ring is idle now)
+  float* mrg = reinterpret_cast<float*>(tiles);        // [kWarps][g][PS]
+  {
+    float l = l_run;
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (qrow < g) {
+      float* rowp = mrg + ((size_t)warp * g + qrow) * PS;
+#pragma unroll
+      for (int n = 0; n < 16; ++n) { rowp[n * 8 + qcol] = o[n][0]; rowp[n * 8 + qcol + 1] = o[n][1]; }
+      if ((lane & 3) == 0) { rowp[kD] = m_run; rowp[kD + 1] = l; }
+    }
+  }
+  __syncthreads();
+  float* my_part = part + ((size_t)sl * splits + split) * g * PS;
+  for (int i = tid; i < g * kD; i += kThreads) {
+    const int h = i / kD, c = i % kD;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mrg[((size_t)w * g + h) * PS + kD]);
+    float acc = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float* rowp = mrg + ((size_t)w * g + h) * PS;
+      const float f = rowp[kD] == -INFINITY ? 0.f : exp2f(rowp[kD] - M);
+      acc = fmaf(rowp[c], f, acc);
+      L = fmaf(rowp[kD + 1], f, L);
+    }
+    my_part[h * PS + c] = acc;
+    if (c == 0) { my_part[h * PS + kD] = M; my_part[h * PS + kD + 1] = L; }
+  }
+  // ---- ticket: the last CTA of the stream combines the splits
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned old = atomicAdd(&tickets[sl], 1u);
+    is_last_s = old == (unsigned)(splits - 1);
+  }
+  __syncthreads();
+  if (!is_last_s) return;
+  __threadfence();
+  const float* sp = part + (size_t)sl * splits * g * PS;
+  for (int i = tid; i < g * kD; i += kThreads) {
+    const int h = i / kD, c = i % kD;
+    float M = -INFINITY;
+    for (int s = 0; s < splits; ++s) M = fmaxf(M, __ldcg(sp + ((size_t)s * g + h) * PS + kD));
+    float acc = 0.f, L = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float* rowp = sp + ((size_t)s * g + h) * PS;
+      const float ms = __ldcg(rowp + kD);
+      const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+      acc = fmaf(__ldcg(rowp + c), f, acc);
+      L = fmaf(__ldcg(rowp + kD + 1), f, L);
+    }
+    out[((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  }
+  if (tid == 0) tickets[sl] = 0;   // ready for the next launch
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kStages * sizeof(uint64_t);
+
+}  // namespace
+
+bool decode_mma_supported(const Geom& G) { return G.is_bf16 && G.d == kD && G.g <= 8; }
+
+// Tensor maps over the K and V arenas viewed as [total_rows, 128] bf16, boxes of 64 dims x 64 rows.
+cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out) {
+  *maps_out = nullptr;
+  if (!decode_mma_supported(G) || total_rows >= ((int64_t)1 << 31)) return cudaErrorNotSupported;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+  DecodeMaps* tm = new DecodeMaps();
+  const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)total_rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kTN};
+  const cuuint32_t estr[2] = {1, 1};
+  void* bases[2] = {A.K, A.V};
+  CUtensorMap* maps[2] = {&tm->k, &tm->v};
+  for (int i = 0; i < 2; ++i) {
+    CUresult r = encode(maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[i], dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { delete tm; return cudaErrorInvalidValue; }
+  }
+  e = cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (e != cudaSuccess) { delete tm; return e; }
+  *maps_out = tm;
+  return cudaSuccess;
+}
+
+void decode_mma_release(void* maps) { delete static_cast<DecodeMaps*>(maps); }
+
+// Same scratch layout as launch_decode: ticket counters, then (stream, split, head) partial rows.
+cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
+                              int splits, int* status, const void* maps, cudaStream_t st) {
+  if (!maps) return cudaErrorInvalidValue;
+  const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
+  const int n_sl = G.B * G.H;
+  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
+  float* part = scratch + ((n_sl + 63) / 64) * 64;
+  dim3 grid(n_sl, splits);
+  decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q),
+                                                        static_cast<__nv_bfloat16*>(out), part, tickets, status, tm->k,
+                                                        tm->v);
+  return cudaGetLastError();
+}
+
+}  // namespace bkv
