@@ -61,7 +61,7 @@ typedef struct balancekv_config {
   int32_t gram_path;     /* 0 = automatic, 1 = CUDA-core (fp32 FMA) kernels for the walk and for
                             decode, 2 = tensor-core (tcgen05) walk kernel; 2 needs bf16,
                             d = 128, t multiple of 128                                         */
-  int32_t reserved;
+  int32_t decode_splits; /* > 0: split-K factor of decode attention (1..64); 0 = automatic         */
   uint64_t seed;         /* Philox key; sequence s uses seed + s                              */
   float delta;           /* failure probability of Algorithm 2; <= 0 means 1/N^2              */
   float c_override;      /* > 0: use this c instead of 30 ln(t/delta)                         */

@@ -41,7 +41,7 @@ class Config(C.Structure):
         ("n_seqs", C.c_int32), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32),
         ("head_dim", C.c_int32), ("dtype", C.c_int32), ("block", C.c_int32), ("levels", C.c_int32),
         ("max_tokens", C.c_int32), ("max_pending", C.c_int32), ("recent_window", C.c_int32),
-        ("center_keys", C.c_int32), ("gram_path", C.c_int32), ("reserved", C.c_int32),
+        ("center_keys", C.c_int32), ("gram_path", C.c_int32), ("decode_splits", C.c_int32),
         ("seed", C.c_uint64), ("delta", C.c_float), ("c_override", C.c_float), ("r_key", C.c_float),
         ("r_value", C.c_float),
     ]
@@ -133,7 +133,7 @@ class Context:
 
     def __init__(self, n_seqs=1, n_layers=1, n_kv_heads=1, n_q_heads=None, head_dim=128, dtype="bf16", block=1024,
                  levels=2, max_tokens=32768, max_pending=0, recent_window=0, center_keys=0, gram_path=0, seed=0,
-                 delta=0.0, c_override=0.0, r_key=0.0, r_value=0.0):
+                 decode_splits=0, delta=0.0, c_override=0.0, r_key=0.0, r_value=0.0):
         import torch
 
         if not torch.cuda.is_available():
@@ -141,7 +141,7 @@ class Context:
         self.lib = load()
         self.cfg = Config(n_seqs, n_layers, n_kv_heads, n_q_heads if n_q_heads else n_kv_heads, head_dim,
                           1 if dtype == "bf16" else 0, block, levels, max_tokens, max_pending, recent_window,
-                          center_keys, gram_path, 0, seed, delta, c_override, r_key, r_value)
+                          center_keys, gram_path, decode_splits, seed, delta, c_override, r_key, r_value)
         self.dtype = _torch_dtype(self.cfg.dtype)
         self._h = C.c_void_p()
         _check(self.lib.balancekv_create(C.byref(self.cfg), C.byref(self._h)), "balancekv_create")

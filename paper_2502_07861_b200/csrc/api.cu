@@ -167,6 +167,7 @@ int check_config(const balancekv_config& f) {
   if (f.levels < 0 || f.levels > kMaxLevels) return BALANCEKV_E_INVAL;
   if (f.max_tokens < 1 || f.recent_window < 0) return BALANCEKV_E_INVAL;
   if (f.gram_path < 0 || f.gram_path > 2) return BALANCEKV_E_INVAL;
+  if (f.decode_splits < 0 || f.decode_splits > 64) return BALANCEKV_E_INVAL;
   return BALANCEKV_OK;
 }
 
@@ -281,6 +282,7 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   {
     const int n_sl = f.n_seqs * f.n_kv_heads;
     c->max_splits = std::max(1, std::min(64, (2 * c->sm_count + n_sl - 1) / n_sl));
+    if (f.decode_splits > 0) c->max_splits = std::min(64, f.decode_splits);
     const size_t sb = decode_scratch_bytes(G, c->max_splits);
     if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->d_decode_scratch), sb))) return fail(rc);
     if (cudaMemset(c->d_decode_scratch, 0, sb) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
@@ -565,7 +567,8 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
     }
   const int tile_tokens = 16384 / (f.head_dim * c->esz);
   const int64_t tiles = (max_rows + tile_tokens - 1) / tile_tokens + f.levels;
-  const int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
+  int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
+  if (f.decode_splits > 0) splits = std::min(f.decode_splits, c->max_splits);
   {
     ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
     if (c->decode_maps)

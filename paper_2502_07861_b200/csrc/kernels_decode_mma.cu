@@ -33,7 +33,7 @@ constexpr uint32_t kHalf = kTN * 128;        // bytes of one [64 tokens][64 dims
 constexpr uint32_t kTensorBytes = 2 * kHalf; // K (or V) tile: two boxes
 constexpr uint32_t kStageBytes = 2 * kTensorBytes;
 constexpr long long kWaitCycles = 4000000000LL;
-constexpr int PS = kD + 2;                   // partial row: acc[D], max, sum
+constexpr int PS = kD + 4;                   // partial row: acc[D], max, sum, 2 pad (rows stay 16-byte aligned)
 
 struct DecodeMaps {
   CUtensorMap k, v;
@@ -288,20 +288,52 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   __syncthreads();
   if (!is_last_s) return;
   __threadfence();
+  // Combine: first the (max, sum) pairs of all splits in one round of loads, then every thread
+  // sums its output columns over the splits with independent loads.
   const float* sp = part + (size_t)sl * splits * g * PS;
-  for (int i = tid; i < g * kD; i += kThreads) {
-    const int h = i / kD, c = i % kD;
-    float M = -INFINITY;
-    for (int s = 0; s < splits; ++s) M = fmaxf(M, __ldcg(sp + ((size_t)s * g + h) * PS + kD));
-    float acc = 0.f, L = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      const float* rowp = sp + ((size_t)s * g + h) * PS;
-      const float ms = __ldcg(rowp + kD);
-      const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-      acc = fmaf(__ldcg(rowp + c), f, acc);
-      L = fmaf(__ldcg(rowp + kD + 1), f, L);
+  float* cm = reinterpret_cast<float*>(tiles);            // [splits][g] max, later the scale factors
+  float* cl = cm + 64 * kMaxGroup;                        // [splits][g] sums
+  float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
+  float* cL = cM + kMaxGroup;                             // [g] overall sum
+  for (int i = tid; i < splits * g; i += kThreads) {
+    const float* rowp = sp + (size_t)i * PS;
+    cm[i] = __ldcg(rowp + kD);
+    cl[i] = __ldcg(rowp + kD + 1);
+  }
+  __syncthreads();
+  for (int h = warp; h < g; h += kWarps) {     // one warp per head, lanes over the (<= 64) splits
+    const int s0 = lane, s1 = lane + 32;
+    const float m0 = s0 < splits ? cm[s0 * g + h] : -INFINITY, m1 = s1 < splits ? cm[s1 * g + h] : -INFINITY;
+    const float M = warp_max(fmaxf(m0, m1));
+    const float f0 = m0 == -INFINITY ? 0.f : exp2f(m0 - M), f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M);
+    float L = (s0 < splits ? cl[s0 * g + h] * f0 : 0.f) + (s1 < splits ? cl[s1 * g + h] * f1 : 0.f);
+    L = warp_sum(L);
+    if (s0 < splits) cm[s0 * g + h] = f0;
+    if (s1 < splits) cm[s1 * g + h] = f1;
+    if (lane == 0) { cM[h] = M; cL[h] = L; }
+  }
+  __syncthreads();
+  // every thread owns 4 consecutive output columns of one head; 8 splits' loads in flight
+  for (int i = tid; i < g * (kD / 4); i += kThreads) {
+    const int h = i / (kD / 4), c = (i % (kD / 4)) * 4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < splits; s += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        v[u] = s + u < splits ? __ldcg(reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c))
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float f = s + u < splits ? cm[(s + u) * g + h] : 0.f;
+        acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
+        acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+      }
     }
-    out[((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+    const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
+    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c);
+    o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
   }
   if (tid == 0) tickets[sl] = 0;   // ready for the next launch
 }
