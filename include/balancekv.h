@@ -192,9 +192,14 @@ int balancekv_reset(balancekv_ctx* ctx, void* stream);
  * writes, per class, {launches, total milliseconds} into out_host[2*class + {0,1}], then
  * clears the record.  Classes: 0 append/load, 1 radii (inputs of Algorithm 2), 2 Gram tiles +
  * sign walk (Algorithm 2), 3 strict-half selection + compaction, 4 decode attention
- * (Algorithm 1's output ratio), 5 bookkeeping (remainder move, segment table). */
+ * (Algorithm 1's output ratio), 5 bookkeeping (remainder move, segment table).
+ * `on`: 0 = off, 1 = every class, any other value = a mask with bit (1 + class) set for each
+ * class to time.  balancekv_profile_sample makes the record of one class sparse: only every
+ * `every`-th launch of it (counted from the call) is timed, which keeps the events out of the
+ * way of a loop of microsecond-sized launches; read then reports the timed launches only. */
 #define BALANCEKV_PROFILE_CLASSES 6
 int balancekv_profile_enable(balancekv_ctx* ctx, int on);
+int balancekv_profile_sample(balancekv_ctx* ctx, int kernel_class, int every);
 int balancekv_profile_read(balancekv_ctx* ctx, double* out_host);
 
 int balancekv_stats(balancekv_ctx* ctx, balancekv_stats_t* out);

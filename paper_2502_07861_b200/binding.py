@@ -21,7 +21,7 @@ EXPORTS = [
     "balancekv_decode_attn", "balancekv_decode_attn_host", "balancekv_cache_load_level",
     "balancekv_cache_view", "balancekv_level_sizes", "balancekv_debug_enable", "balancekv_debug_call",
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
-    "balancekv_profile_enable", "balancekv_profile_read", "balancekv_decode_attn_static",
+    "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
@@ -85,6 +85,7 @@ def load():
     lib.balancekv_stream_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.balancekv_stream_step_host.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.balancekv_profile_enable.argtypes = [vp, ci]
+    lib.balancekv_profile_sample.argtypes = [vp, ci, ci]
     lib.balancekv_profile_read.argtypes = [vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     for name in EXPORTS:
@@ -277,8 +278,17 @@ class Context:
     def reset(self, stream=None):
         _check(self.lib.balancekv_reset(self._h, _stream_ptr(stream)), "balancekv_reset")
 
-    def profile_enable(self, on=True):
-        _check(self.lib.balancekv_profile_enable(self._h, 1 if on else 0), "balancekv_profile_enable")
+    def profile_enable(self, on=True, classes=None):
+        """Time every kernel class, or only the named ones (see PROFILE_CLASSES)."""
+        flag = 1 if on else 0
+        if on and classes is not None:
+            flag = sum(2 << PROFILE_CLASSES.index(n) for n in classes)
+        _check(self.lib.balancekv_profile_enable(self._h, flag), "balancekv_profile_enable")
+
+    def profile_sample(self, kernel_class, every):
+        """Time only every `every`-th launch of one class (name from PROFILE_CLASSES)."""
+        _check(self.lib.balancekv_profile_sample(self._h, PROFILE_CLASSES.index(kernel_class), int(every)),
+               "balancekv_profile_sample")
 
     def profile_read(self):
         """{class name: (launches, total ms)} since the last read."""

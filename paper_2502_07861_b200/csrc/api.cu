@@ -92,7 +92,9 @@ struct balancekv_ctx {
   std::vector<std::vector<int>> layer_stream_ids;
 
   // optional per-class kernel timing
-  bool profiling = false;
+  unsigned profiling = 0;                   // bit per kernel class
+  int prof_every[BALANCEKV_PROFILE_CLASSES] = {1, 1, 1, 1, 1, 1};
+  unsigned long long prof_seen[BALANCEKV_PROFILE_CLASSES] = {0, 0, 0, 0, 0, 0};
   std::vector<cudaEvent_t> prof_ev;     // pairs
   std::vector<int> prof_class;
   size_t prof_used = 0;
@@ -104,7 +106,7 @@ constexpr size_t kProfMax = 8192;
 struct ProfScope {
   balancekv_ctx* c; cudaStream_t st; bool on;
   ProfScope(balancekv_ctx* c_, int cls, cudaStream_t st_) : c(c_), st(st_), on(false) {
-    if (c->profiling && c->prof_used < kProfMax) {
+    if (((c->profiling >> cls) & 1u) && c->prof_seen[cls]++ % c->prof_every[cls] == 0 && c->prof_used < kProfMax) {
       on = true;
       c->prof_class[c->prof_used] = cls;
       cudaEventRecord(c->prof_ev[2 * c->prof_used], st);
@@ -720,7 +722,14 @@ int balancekv_profile_enable(balancekv_ctx* c, int on) {
     c->prof_class.resize(kProfMax);
     for (cudaEvent_t& e : c->prof_ev) BKV_CUDA(cudaEventCreate(&e));
   }
-  c->profiling = on != 0;
+  c->profiling = on == 1 ? ~0u : static_cast<unsigned>(on) >> 1;   // bit `class` set: time that class
+  return BALANCEKV_OK;
+}
+
+int balancekv_profile_sample(balancekv_ctx* c, int cls, int every) {
+  if (!c || cls < 0 || cls >= BALANCEKV_PROFILE_CLASSES || every < 1) return BALANCEKV_E_INVAL;
+  c->prof_every[cls] = every;
+  c->prof_seen[cls] = 0;
   return BALANCEKV_OK;
 }
 
