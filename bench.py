@@ -176,6 +176,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2502_07861_b200 as bk
+    from paper_2502_07861_b200 import shard
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -204,7 +205,7 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     ctx = bk.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, head_dim=d, dtype="bf16", block=t, levels=T,
-                     max_tokens=n_ctx + n_dec, seed=w["walk_seed"] + rank, gram_path=args.gram_path)
+                     max_tokens=n_ctx + n_dec, seed=shard.walk_seed(w["walk_seed"], rank * B), gram_path=args.gram_path)
 
     raw_stream = int(torch.cuda.current_stream().cuda_stream)
     q_list, K_list, V_list = list(q_d.unbind(0)), list(K_dec.unbind(0)), list(V_dec.unbind(0))
@@ -259,10 +260,7 @@ def main():
     t_comp = np.array([e[0].elapsed_time(e[1]) for e in evs])
     t_dec = np.array([e[1].elapsed_time(e[2]) for e in evs])
     total_ms = float(t_step.sum())
-    if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = shard.max_over_ranks(total_ms, device="cuda")
     units_per_step = B * H * n_ctx
     value = world * units_per_step * args.steps / (total_ms * 1e-3)
 
@@ -276,10 +274,7 @@ def main():
         step_host()
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        tt = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_s = float(tt.item())
+    e2e_s = shard.max_over_ranks(e2e_s, device="cuda")
     esz = 2
     h2d = 2 * B * H * (n_ctx + n_dec) * d * esz + n_dec * B * Hq * d * esz
     d2h = n_dec * B * Hq * d * esz
