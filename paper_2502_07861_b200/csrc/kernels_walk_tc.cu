@@ -4,20 +4,26 @@
 //   Ghat_ij = exp((<k_i,k_j> - r_key^2)/sqrt d) <v_i,v_j> / r_value^2      (proof of Theorem 3.2)
 // is visited in 128 x 128 tiles of its lower triangle, row panel by row panel.  For a tile,
 // TMA brings the bf16 rows of K and V into 128B-swizzled shared memory, tcgen05.mma
-// (bf16 x bf16 -> fp32) forms K_r K_c^T and V_r V_c^T in two TMEM accumulators, and two
-// epilogue warpgroups (thread = row, 64 columns of the tile each) read them back with
+// (bf16 x bf16 -> fp32) forms K_r K_c^T and V_r V_c^T in two TMEM accumulators, and four
+// epilogue warpgroups (thread = row, 32 columns of the tile each) read them back with
 // tcgen05.ld, apply exp2/scale/product and fold the tile into the row's running correlation
 //   S_j = sum_{i<j} eta_i Ghat_ij
-// with the signs of earlier panels.  The diagonal tile feeds the walk: warp q owns rows
-// 32q..32q+31 of the panel, lane l owns one token,
+// with the signs of earlier panels.  The diagonal tile feeds the walk,
 //   eta_j = +1  iff  u_j < 1/2 - S_j/(2c)  <=>  S_j < c (1 - 2 u_j),
-// u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).  Inside a 32-token
-// group the sequential recurrence is solved by sweeps (decide all tokens from the current
-// signs, repeat until nothing changes), which reaches exactly the sequential result.
+// u_j the Philox uniform of (seed, layer, head, call ordinal, level, j).  eta_j depends only on
+// eta_{<j}, so the sequential recurrence has a unique solution, and it is the fixed point of
+// "decide every token of the panel from the current signs": all 512 epilogue threads keep their
+// 32 entries of the diagonal tile in registers and repeat that sweep (two named-barrier exchanges
+// per sweep) until no sign changes.  Sweep k makes at least token k final, so 129 sweeps always
+// suffice; with small Ghat two or three do.
 // TMEM is double buffered (2 x 256 columns); an epilogue hands its buffer back as soon as the
 // accumulator values are in registers.  Each of the two products of a tile has its own issuing
 // thread and its own barriers, so that one product's waits and commits overlap the other's
-// MMAs.  Ghat never touches global memory.
+// MMAs.  Operands live in three 64 KB slots (K tile + V tile) that rotate roles: panel r keeps
+// its rows in slot r % 3 and streams its column tiles through the other two, and the rows of
+// panel r + 1 are fetched into the slot that panel r's column tiles leave first, so the next
+// panel's first products are already in TMEM when the walk of the diagonal tile ends.
+// Ghat never touches global memory.
 //
 // Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
 // roles leave their loops, TMEM is freed and the kernel returns.
@@ -30,8 +36,10 @@ namespace bkv {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kThreads = 352;              // warps 0-3, 4-7: two epilogue + walk warpgroups, 8: TMA, 9: MMA (K K^T), 10: MMA (V V^T)
-constexpr int kTmaWarp = 8, kMmaWarp = 9, kMmaWarpV = 10;
+constexpr int kEpiGroups = 4;              // epilogue + walk warpgroups: warps 0-15 (warp % 4 = TMEM lane quadrant)
+constexpr int kEpiWarps = 4 * kEpiGroups;
+constexpr int kTmaWarp = kEpiWarps, kMmaWarp = kEpiWarps + 1, kMmaWarpV = kEpiWarps + 2;   // TMA, MMA (K K^T), MMA (V V^T)
+constexpr int kThreads = 32 * (kEpiWarps + 3);
 constexpr uint32_t kHalfBytes = 16384;     // [128 rows][64 bf16] = one swizzle-atom column of a tile
 constexpr uint32_t kTileBytes = 32768;     // [128 rows][128 bf16]
 constexpr uint32_t kTmemCols = 512;
@@ -79,15 +87,20 @@ __device__ inline bool wait_bar(uint64_t* bar, uint32_t parity, int* abort_flag)
   }
   return true;
 }
-// Bounded wait until *progress >= need.
-__device__ inline bool wait_progress(const int* progress, int need, int* abort_flag) {
-  if (ld_acquire(progress) >= need) return true;
-  const long long t0 = clock64();
-  while (ld_acquire(progress) < need) {
-    if (ld_acquire(abort_flag)) return false;
-    if (clock64() - t0 > kWaitCycles) { st_release(abort_flag, 1); return false; }
-  }
-  return true;
+// Named barriers of the 512 epilogue threads (ids 1..3; id 0 is __syncthreads).  Every epilogue
+// thread reaches every one of them whatever happened before (a failed wait only clears `ok`), so
+// none of them can be left waiting.
+__device__ inline void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ inline void bar_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ inline bool bar_red_or(int id, int n, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(id), "r"(n), "r"((uint32_t)pred) : "memory");
+  return r != 0;
 }
 
 __device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -187,13 +200,14 @@ __device__ inline float2 poly_exp2x2(float2 x) {
 }
 // Of the 16 column pairs of a 32-column chunk, pairs with (index % 8) < kPolyOf8 take the
 // polynomial path, the others the special-function unit.
-constexpr int kPolyOf8 = 3;
+constexpr int kPolyOf8 = 1;
 
 struct Smem {
-  // operand tiles first (1024-byte aligned for the 128B swizzle)
-  static constexpr uint32_t kKr = 0, kVr = kTileBytes, kStage0 = 2 * kTileBytes;   // stage: K then V
-  static constexpr uint32_t kTilesEnd = 6 * kTileBytes;
+  // three operand slots first (1024-byte aligned for the 128B swizzle); a slot holds a K tile then a V tile
+  static constexpr uint32_t kSlotBytes = 2 * kTileBytes;
+  static constexpr uint32_t kTilesEnd = 3 * kSlotBytes;
 };
+constexpr int kMaxSweeps = kTile + 2;
 
 template <bool kCenter>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -205,35 +219,32 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int t = G.t, P = t / kTile;
-  float* etas = reinterpret_cast<float*>(sm + Smem::kTilesEnd);          // [t] signs scaled by 1/r_value^2
-  float* xacc = etas + t;                                                 // [2][128] partial correlations handed over
-  int8_t* eta8 = reinterpret_cast<int8_t*>(xacc + 2 * kTile);             // [t] signs
+  float* etas = reinterpret_cast<float*>(sm + Smem::kTilesEnd);          // [t] signs scaled by 1/r_value^2 (0 = undecided)
+  float* xs = etas + t;                                                   // [3][128] partial correlations of column quarters 1..3
+  float* thr_s = xs + (kEpiGroups - 1) * kTile;                           // [t] decision thresholds c (1 - 2 u_j)
+  int8_t* eta8 = reinterpret_cast<int8_t*>(thr_s + t);                    // [t] signs
   uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
   // x = 0: the K K^T product, x = 1: the V V^T product
-  uint64_t* row_full = bars + 0;     // row panel landed
-  uint64_t* xfull = bars + 1;        // [x][2] column tile of product x landed in stage s
-  uint64_t* xdone = bars + 5;        // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
-  uint64_t* xcempty = bars + 9;      // [x][2] product x no longer reads column stage s -> producer
-  uint64_t* xrempty = bars + 13;     // [x]    product x no longer reads the row panel -> producer
-  uint64_t* tmem_empty = bars + 15;  // [2] both warpgroups have drained buffer b
-  uint64_t* xacc_full = bars + 17;   // [2][4]: per panel parity and warp quarter
-  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 25);
-  int* progress = reinterpret_cast<int*>(tmem_ptr_s + 1);
-  int* abort_flag = progress + 1;
+  uint64_t* full = bars + 0;         // [x][3] operand tile of product x landed in slot s
+  uint64_t* empty = bars + 6;        // [x][3] product x no longer reads slot s -> producer
+  uint64_t* xdone = bars + 12;       // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
+  uint64_t* tmem_empty = bars + 16;  // [2] both warpgroups have drained buffer b
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 18);
+  int* abort_flag = reinterpret_cast<int*>(tmem_ptr_s + 1);
 
   const int call = blockIdx.x;
   const CallDesc C = calls[call];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
-    mbar_init(row_full, 1);
-    for (int i = 0; i < 4; ++i) { mbar_init(xfull + i, 1); mbar_init(xdone + i, 1); mbar_init(xcempty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(xrempty + i, 1); mbar_init(tmem_empty + i, 256); }
-    for (int i = 0; i < 8; ++i) mbar_init(xacc_full + i, 32);
-    *progress = 0; *abort_flag = 0;
+    for (int i = 0; i < 6; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); }
+    for (int i = 0; i < 4; ++i) mbar_init(xdone + i, 1);
+    for (int i = 0; i < 2; ++i) mbar_init(tmem_empty + i, kEpiWarps);       // one arrival per warp (lane 0 after __syncwarp)
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  for (int i = tid; i < t; i += kThreads) etas[i] = 0.f;
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_ptr_s)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -244,41 +255,38 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   const uint32_t tmem_base = *tmem_ptr_s;
 
   // Tiles are numbered in issue order i = 0, 1, ...: panel r contributes (r,0) .. (r,r).  Tile i
-  // uses TMEM buffer i & 1 and, unless it is a diagonal tile, column stage i & 1.  Every barrier
-  // is waited on phase by phase by its one kind of waiter, and each next phase depends on that
-  // waiter having passed, so a parity wait can never be a phase behind.
+  // uses TMEM buffer i & 1.  Panel r reads its rows from slot r % 3 and column tile c from slot
+  // (r + 1 + (c & 1)) % 3.  Loads happen in the order R0, R1, C(1,0), R2, C(2,0), C(2,1), R3, ...
+  // (R = row panel), which is also the order in which the MMA threads first touch them, so both
+  // sides count the uses of a slot alike.  Every barrier is waited on phase by phase by its one
+  // kind of waiter, and each next phase depends on that waiter having passed, so a parity wait
+  // can never be a phase behind.
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int i = 0, use0 = 0, use1 = 0;      // tiles so far; column tiles that used stage 0 / 1
+      uint32_t used = 0, par = 0;        // per slot: loaded before; parity of the next wait on its empty barriers
       bool ok = true;
+      auto load = [&](int slot, int tile_row) -> bool {
+        const bool again = (used >> slot) & 1u;
+        const uint32_t ph = (par >> slot) & 1u;
+        used |= 1u << slot;
+        if (again) par ^= 1u << slot;
+        unsigned char* st = sm + (uint32_t)slot * Smem::kSlotBytes;
+        const int y = (int)(C.src_row + (int64_t)tile_row * kTile);
+        if (again && !wait_bar(empty + slot, ph, abort_flag)) return false;
+        mbar_expect_tx(full + slot, kTileBytes);
+        tma_load_2d(st, &tmK, 0, y, full + slot);
+        tma_load_2d(st + kHalfBytes, &tmK, 64, y, full + slot);
+        if (again && !wait_bar(empty + 3 + slot, ph, abort_flag)) return false;
+        mbar_expect_tx(full + 3 + slot, kTileBytes);
+        tma_load_2d(st + kTileBytes, &tmV, 0, y, full + 3 + slot);
+        tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, y, full + 3 + slot);
+        return true;
+      };
+      ok = load(0, 0);
       for (int r = 0; r < P && ok; ++r) {
-        if (r > 0) {   // both products have finished the previous panel's diagonal tile
-          if (!(ok = wait_bar(xrempty + 0, (uint32_t)((r - 1) & 1), abort_flag))) break;
-          if (!(ok = wait_bar(xrempty + 1, (uint32_t)((r - 1) & 1), abort_flag))) break;
-        }
-        const int y = (int)(C.src_row + (int64_t)r * kTile);
-        mbar_expect_tx(row_full, 2 * kTileBytes);
-        tma_load_2d(sm + Smem::kKr, &tmK, 0, y, row_full);
-        tma_load_2d(sm + Smem::kKr + kHalfBytes, &tmK, 64, y, row_full);
-        tma_load_2d(sm + Smem::kVr, &tmV, 0, y, row_full);
-        tma_load_2d(sm + Smem::kVr + kHalfBytes, &tmV, 64, y, row_full);
-        for (int c = 0; c < r; ++c, ++i) {
-          const int s = i & 1;
-          const int n = s ? use1 : use0;                              // earlier users of this stage
-          if (s) ++use1; else ++use0;
-          unsigned char* st = sm + Smem::kStage0 + (uint32_t)s * 2 * kTileBytes;
-          const int yc = (int)(C.src_row + (int64_t)c * kTile);
-          if (n > 0 && !(ok = wait_bar(xcempty + s, (uint32_t)((n - 1) & 1), abort_flag))) break;
-          mbar_expect_tx(xfull + s, kTileBytes);
-          tma_load_2d(st, &tmK, 0, yc, xfull + s);
-          tma_load_2d(st + kHalfBytes, &tmK, 64, yc, xfull + s);
-          if (n > 0 && !(ok = wait_bar(xcempty + 2 + s, (uint32_t)((n - 1) & 1), abort_flag))) break;
-          mbar_expect_tx(xfull + 2 + s, kTileBytes);
-          tma_load_2d(st + kTileBytes, &tmV, 0, yc, xfull + 2 + s);
-          tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, yc, xfull + 2 + s);
-        }
-        ++i;   // the diagonal tile loads nothing
+        for (int c = 0; c < r && ok; ++c) ok = load((r + 1 + (c & 1)) % 3, c);
+        if (ok && r + 1 < P) ok = load((r + 1) % 3, r + 1);
       }
     }
     __syncwarp();
@@ -286,55 +294,59 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     // ------------------------------------------------------------------ MMA issuers (K K^T and V V^T)
     if (lane == 0) {
       const int x = warp == kMmaWarpV ? 1 : 0;
-      int i = 0, use0 = 0, use1 = 0;
+      int i = 0;
+      uint32_t par = 0;                  // per slot: parity of the next wait on its full barrier
       bool ok = true;
-      const uint32_t arow = umma_desc_lo(smem_u32(sm + (x ? Smem::kVr : Smem::kKr)));
-      const uint32_t st0 = umma_desc_lo(smem_u32(sm + Smem::kStage0 + (x ? kTileBytes : 0u)));
+      const uint32_t slot0 = umma_desc_lo(smem_u32(sm + (x ? kTileBytes : 0u)));
+      constexpr uint32_t kSlotDesc = Smem::kSlotBytes >> 4;
       for (int r = 0; r < P && ok; ++r) {
-        if (!(ok = wait_bar(row_full, (uint32_t)(r & 1), abort_flag))) break;
+        const int rs = r % 3;
+        if (!(ok = wait_bar(full + 3 * x + rs, (par >> rs) & 1u, abort_flag))) break;
+        par ^= 1u << rs;
+        const uint32_t arow = slot0 + (uint32_t)rs * kSlotDesc;
         for (int c = 0; c <= r; ++c, ++i) {
           const int buf = i & 1;
           if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag))) break;
           uint32_t b = arow;
+          int slot = rs;
           if (c < r) {
-            const int n = buf ? use1 : use0;
-            if (buf) ++use1; else ++use0;
-            if (!(ok = wait_bar(xfull + 2 * x + buf, (uint32_t)(n & 1), abort_flag))) break;
-            b = st0 + (uint32_t)buf * ((2 * kTileBytes) >> 4);
+            slot = (r + 1 + (c & 1)) % 3;
+            if (!(ok = wait_bar(full + 3 * x + slot, (par >> slot) & 1u, abort_flag))) break;
+            par ^= 1u << slot;
+            b = slot0 + (uint32_t)slot * kSlotDesc;
           }
           tc_fence_after();
           umma_tile(tmem_base + (uint32_t)buf * 256u + (x ? 128u : 0u), arow, b);
-          if (c < r) umma_commit(xcempty + 2 * x + buf);
-          else umma_commit(xrempty + x);
+          umma_commit(empty + 3 * x + slot);     // a column slot after its tile, the row slot after the diagonal tile
           umma_commit(xdone + 2 * x + buf);
         }
       }
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ two epilogue warpgroups
-    // Every tile is drained by both warpgroups: group wg takes columns 64 wg .. 64 wg + 63 of the
-    // tile (thread = row).  Each thread keeps a partial running correlation of its row; at the
-    // diagonal tile the panel's owner group (alternating) collects the other group's partial and
-    // walks the panel, while the other group folds in the diagonal tile's older columns.
+    // ------------------------------------------------------------------ four epilogue warpgroups
+    // Every tile is drained by all groups: group wg takes columns 32 wg .. 32 wg + 31 of the tile
+    // (thread = row) and keeps a partial running correlation of its row over those columns.
     const int wg = warp >> 2;
     const int q = warp & 3;                   // quarter of the panel = TMEM lane quadrant
     const int row = 32 * q + lane;
-    const int head = C.stream % G.H;
-    const int layer = (C.stream / G.H) % G.L;
-    const int seq = C.stream / (G.H * G.L);
     const float rk2 = G.fixed_rk2 > 0.f ? G.fixed_rk2 : stats[call].rk2;
     const float rv2 = G.fixed_rv2 > 0.f ? G.fixed_rv2 : stats[call].rv2;
     const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
     const float scale = 1.4426950408889634f * G.inv_sqrt_d;
     const float cw = G.c;
-    const uint32_t tlane = tmem_base + ((uint32_t)(32 * q) << 16);
+    const uint32_t tlane = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * wg);
     const float* shift = kCenter ? tok_shift + (size_t)call * t : nullptr;
     int tile_it = 0, fails = 0;
     bool ok = true;
 
-    // acc += sum over 32 columns of Ghat' * sign, from accumulator values already in registers;
-    // two columns at a time with packed fp32 instructions
+    // Ghat' (without 1/r_value^2) of two neighbouring columns, packed fp32
+    auto ghat2 = [&](float k0, float k1, float v0, float v1, float nb, bool poly) -> float2 {
+      const float2 ex = __ffma2_rn(make_float2(k0, k1), make_float2(scale, scale), make_float2(nb, nb));
+      const float2 ee = poly ? poly_exp2x2(ex) : make_float2(fast_exp2(ex.x), fast_exp2(ex.y));
+      return __fmul2_rn(ee, make_float2(v0, v1));
+    };
+    // acc += sum over this group's 32 columns of Ghat' * sign, from accumulator values in registers
     auto fold_regs = [&](const float (&dk)[32], const float (&dv)[32], const float* signs, int shift_base, float nb,
                          float acc) -> float {
       const float4* e4 = reinterpret_cast<const float4*>(signs);
@@ -352,157 +364,133 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
         }
         return acc;
       } else {
-        float2 acc2 = make_float2(acc, 0.f);
-        const float2 sc2 = make_float2(scale, scale), nb2 = make_float2(nb, nb);
+        float2 a2[2] = {make_float2(acc, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
           const float4 e = e4[x];
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const int i = 4 * x + 2 * h, pair = 2 * x + h;
-            const float2 ex = __ffma2_rn(make_float2(dk[i], dk[i + 1]), sc2, nb2);
-            float2 ee;
-            if ((pair & 7) < kPolyOf8) ee = poly_exp2x2(ex);
-            else ee = make_float2(fast_exp2(ex.x), fast_exp2(ex.y));
-            const float2 g = __fmul2_rn(ee, make_float2(dv[i], dv[i + 1]));
-            acc2 = __ffma2_rn(g, h ? make_float2(e.z, e.w) : make_float2(e.x, e.y), acc2);
+            const float2 g = ghat2(dk[i], dk[i + 1], dv[i], dv[i + 1], nb, (pair & 7) < kPolyOf8);
+            a2[pair & 1] = __ffma2_rn(g, h ? make_float2(e.z, e.w) : make_float2(e.x, e.y), a2[pair & 1]);
           }
         }
-        return acc2.x + acc2.y;
+        const float2 s2 = __fadd2_rn(a2[0], a2[1]);
+        return s2.x + s2.y;
       }
     };
-    auto fold_chunk = [&](uint32_t tb, int ch, const float* signs, int shift_base, float nb, float acc) -> float {
-      float dk[32], dv[32];
-      tmem_ld32(tb + ch * 32, dk);
-      tmem_ld32(tb + 128 + ch * 32, dv);
-      tmem_ld_wait();
-      return fold_regs(dk, dv, signs + ch * 32, shift_base + ch * 32, nb, acc);
-    };
 
-    for (int r = 0; r < P && ok; ++r) {
+    constexpr int kEpiThreads = 32 * kEpiWarps;
+    {
+      // all coins of the call up front (the first tile is still on its way), off the walk's critical path
+      const int head = C.stream % G.H, layer = (C.stream / G.H) % G.L, seq = C.stream / (G.H * G.L);
+      for (int i = tid; i < t; i += kEpiThreads)
+        thr_s[i] = cw * (1.0f - 2.0f * walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, i));
+      bar_sync(3, kEpiThreads);
+    }
+    // All waits of a panel come before its vote barrier (id 3); a thread whose wait timed out
+    // skips to the vote, where everybody learns of it and leaves.  The sweep barriers (ids 1, 2)
+    // come after the vote and contain no waits, so no thread can be left waiting at them.
+    for (int r = 0; r < P; ++r) {
       const int j = r * kTile + row;                      // this thread's token in the panel
       float nb = -rk2 * scale;                            // exponent offset of this row
       if constexpr (kCenter) nb -= shift[j] * scale;
       float acc = 0.f;
+      const int col0 = 32 * wg;
+      const bool below = wg <= q;                         // warp-uniform: the warp has columns below the diagonal
       for (int c = 0; c < r && ok; ++c, ++tile_it) {
         const int buf = tile_it & 1;
-        if (!(ok = wait_progress(progress, 4 * c + 4, abort_flag))) break;     // signs of panel c are final
         if (!(ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
         if (!(ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
         tc_fence_after();
         const uint32_t tb = tlane + (uint32_t)buf * 256u;
-        // pull this group's 64 columns of both accumulators into registers and hand the TMEM
+        // pull this group's 32 columns of both accumulators into registers and hand the TMEM
         // buffer back at once; the arithmetic then overlaps the next tiles' MMAs
-        float dk0[32], dv0[32], dk1[32], dv1[32];
-        tmem_ld32(tb + (2 * wg) * 32, dk0);
-        tmem_ld32(tb + 128 + (2 * wg) * 32, dv0);
-        tmem_ld32(tb + (2 * wg + 1) * 32, dk1);
-        tmem_ld32(tb + 128 + (2 * wg + 1) * 32, dv1);
+        float dk[32], dv[32];
+        tmem_ld32(tb, dk);
+        tmem_ld32(tb + 128, dv);
         tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(tmem_empty + buf);
-        acc = fold_regs(dk0, dv0, etas + c * kTile + (2 * wg) * 32, c * kTile + (2 * wg) * 32, nb, acc);
-        acc = fold_regs(dk1, dv1, etas + c * kTile + (2 * wg + 1) * 32, c * kTile + (2 * wg + 1) * 32, nb, acc);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tmem_empty + buf);
+        // signs of panel c are final since its walk
+        acc = fold_regs(dk, dv, etas + c * kTile + 32 * wg, c * kTile + 32 * wg, nb, acc);
       }
-      if (!ok) break;
       // ---- diagonal tile
       const int buf = tile_it & 1;
-      if (!(ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
-      if (!(ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
-      tc_fence_after();
-      const uint32_t tb = tlane + (uint32_t)buf * 256u;
+      if (ok) ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag);
+      if (ok) ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag);
+      if (bar_red_or(3, kEpiThreads, !ok)) { ok = false; break; }          // uniform: everybody walks or everybody leaves
       ++tile_it;
-      if (wg != (r & 1)) {
-        // helper group: columns of the groups two or more before this warp's, then hand over
-        for (int ch = 0; ch + 1 < q && ok; ++ch) {
-          if (!(ok = wait_progress(progress, 4 * r + ch + 1, abort_flag))) break;
-          acc = fold_chunk(tb, ch, etas + r * kTile, r * kTile, nb, acc);
-        }
-        tc_fence_before();
-        mbar_arrive(tmem_empty + buf);
-        if (!ok) break;
-        xacc[(r & 1) * kTile + row] = acc;
-        mbar_arrive(xacc_full + (r & 1) * 4 + q);
-        continue;
-      }
-      // owner group: Ghat of this row against its warp's own 32 tokens and the 32 before them
-      const float u = walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, j);
-      const float thr = cw * (1.0f - 2.0f * u);
-      float own[32], prev[32];
+      float g[32];
       {
+        tc_fence_after();
+        const uint32_t tb = tlane + (uint32_t)buf * 256u;
         float dk[32], dv[32];
-        tmem_ld32(tb + q * 32, dk);
-        tmem_ld32(tb + 128 + q * 32, dv);
+        tmem_ld32(tb, dk);
+        tmem_ld32(tb + 128, dv);
         tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tmem_empty + buf);
+        // Ghat' of this row against the strictly earlier tokens among this group's columns (none
+        // for the warps above the diagonal)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float ex = fmaf(dk[i], scale, nb);
-          if constexpr (kCenter) ex -= shift[r * kTile + q * 32 + i] * scale;
-          own[i] = i < lane ? fast_exp2(ex) * dv[i] * inv_rv2 : 0.f;       // strictly earlier tokens only
+        for (int i = 0; i < 32; i += 2) {
+          float2 v = make_float2(0.f, 0.f);
+          if (below) {
+            if constexpr (kCenter) {
+              v.x = fast_exp2(fmaf(dk[i], scale, nb) - shift[r * kTile + col0 + i] * scale) * dv[i];
+              v.y = fast_exp2(fmaf(dk[i + 1], scale, nb) - shift[r * kTile + col0 + i + 1] * scale) * dv[i + 1];
+            } else {
+              v = ghat2(dk[i], dk[i + 1], dv[i], dv[i + 1], nb, false);
+            }
+          }
+          g[i] = col0 + i < row ? v.x : 0.f;
+          g[i + 1] = col0 + i + 1 < row ? v.y : 0.f;
         }
       }
-      if (q > 0) {
-        float dk[32], dv[32];
-        tmem_ld32(tb + (q - 1) * 32, dk);
-        tmem_ld32(tb + 128 + (q - 1) * 32, dv);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float ex = fmaf(dk[i], scale, nb);
-          if constexpr (kCenter) ex -= shift[r * kTile + (q - 1) * 32 + i] * scale;
-          prev[i] = fast_exp2(ex) * dv[i];
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(tmem_empty + buf);                     // the TMEM buffer is free while we walk
-      // the other group's partial sums for this row
-      if (!(ok = wait_bar(xacc_full + (r & 1) * 4 + q, (uint32_t)((r >> 1) & 1), abort_flag))) break;
-      float S_pre = acc + xacc[(r & 1) * kTile + row];
-      if (q > 0) {
-        if (!(ok = wait_progress(progress, 4 * r + q, abort_flag))) break;     // the 32 tokens just before
-        const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + (q - 1) * 32);
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          const float4 e = e4[x];
-          s0 = fmaf(prev[4 * x + 0], e.x, s0);
-          s1 = fmaf(prev[4 * x + 1], e.y, s1);
-          s2 = fmaf(prev[4 * x + 2], e.z, s2);
-          s3 = fmaf(prev[4 * x + 3], e.w, s3);
-        }
-        S_pre += (s0 + s1) + (s2 + s3);
-      }
-      // The walk over this warp's 32 tokens.  eta_l depends only on eta_{<l}, so the sequential
-      // solution is the unique fixed point of "decide every token from the current signs"; each
-      // sweep makes at least one more leading token final, and a sweep that changes nothing
-      // proves the fixed point.  With small Ghat two sweeps suffice; 32 always do.
-      float S = S_pre;
-      unsigned mask = __ballot_sync(0xffffffffu, S < thr);
+      const float thr = thr_s[j];
+      // The walk over the panel's 128 tokens by sweeps: group 0 owns the decisions, groups 1-3
+      // supply the partial sums of their columns.  Undecided signs are stored as 0.
+      const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + col0);
+      bool plus = false;
+      float S = 0.f;
 #pragma unroll 1
-      for (int sweep = 0; sweep < 33; ++sweep) {
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+        float part = acc;
+        if (below) {
+          float2 a2 = make_float2(acc, 0.f), b2 = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          s0 += (mask >> (i + 0)) & 1u ? own[i + 0] : -own[i + 0];
-          s1 += (mask >> (i + 1)) & 1u ? own[i + 1] : -own[i + 1];
-          s2 += (mask >> (i + 2)) & 1u ? own[i + 2] : -own[i + 2];
-          s3 += (mask >> (i + 3)) & 1u ? own[i + 3] : -own[i + 3];
+          for (int x = 0; x < 8; ++x) {
+            const float4 e = e4[x];
+            a2 = __ffma2_rn(make_float2(g[4 * x], g[4 * x + 1]), make_float2(e.x, e.y), a2);
+            b2 = __ffma2_rn(make_float2(g[4 * x + 2], g[4 * x + 3]), make_float2(e.z, e.w), b2);
+          }
+          part = (a2.x + a2.y) + (b2.x + b2.y);
         }
-        S = S_pre + ((s0 + s1) + (s2 + s3));
-        const unsigned next = __ballot_sync(0xffffffffu, S < thr);
-        if (next == mask) break;
-        mask = next;
+        bool changed = false;
+        if (wg > 0) {
+          xs[(wg - 1) * kTile + row] = part;
+          bar_arrive(1, kEpiThreads);
+        } else {
+          bar_sync(1, kEpiThreads);                       // all partial sums of this sweep are written
+          S = (part + xs[row]) + (xs[kTile + row] + xs[2 * kTile + row]);
+          const bool now = S < thr;
+          changed = sweep == 0 || now != plus;
+          plus = now;
+          etas[j] = plus ? inv_rv2 : -inv_rv2;
+        }
+        if (!bar_red_or(2, kEpiThreads, changed)) break;  // all signs of this sweep are written; any change?
       }
-      const bool plus = (mask >> lane) & 1u;
-      etas[j] = plus ? inv_rv2 : -inv_rv2;
-      eta8[j] = plus ? 1 : -1;
-      if (fabsf(S) > cw) ++fails;                          // FAIL of Algorithm 2: counted; the decision is the clamped one
-      if (C.dbg_off >= 0) {
-        dbg_S[C.dbg_off + j] = S;
-        dbg_p[C.dbg_off + j] = 0.5f - fminf(fmaxf(S, -cw), cw) / (2.0f * cw);
+      if (wg == 0) {
+        eta8[j] = plus ? 1 : -1;
+        if (fabsf(S) > cw) ++fails;                          // FAIL of Algorithm 2: counted; the decision is the clamped one
+        if (C.dbg_off >= 0) {
+          dbg_S[C.dbg_off + j] = S;
+          dbg_p[C.dbg_off + j] = 0.5f - fminf(fmaxf(S, -cw), cw) / (2.0f * cw);
+        }
       }
-      __syncwarp();
-      if (lane == 0) st_release(progress, 4 * r + q + 1);
     }
     fails = (int)__reduce_add_sync(0xffffffffu, (unsigned)fails);
     if (lane == 0 && fails) atomicAdd(fail_count, (unsigned long long)fails);
@@ -525,7 +513,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 5 + 2 * kTile * 4 + 256; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 9 + (kEpiGroups - 1) * kTile * 4 + 256; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
