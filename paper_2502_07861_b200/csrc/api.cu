@@ -20,6 +20,9 @@ void walk_tc_release(void* tmaps);
 bool decode_mma_supported(const Geom& G);
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out);
 void decode_mma_release(void* maps);
+cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
+                                   int splits, int* status, const void* maps, const void* k_new, const void* v_new,
+                                   int rel_row, int idx0, int new_len, cudaStream_t st);
 cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                               int splits, int* status, const void* maps, cudaStream_t st);
 }  // namespace bkv
@@ -555,9 +558,8 @@ int balancekv_compress_layer(balancekv_ctx* c, int layer, int T, void* stream) {
   return compress_streams(c, layer_streams(c, layer), T, static_cast<cudaStream_t>(stream));
 }
 
-int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out, void* stream) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return BALANCEKV_E_INVAL;
-  if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
+// Split-K factor of a decode launch over the layer's current caches.
+static int pick_splits(balancekv_ctx* c, int layer) {
   const balancekv_config& f = c->cfg;
   int64_t max_rows = 0;
   for (int s = 0; s < f.n_seqs; ++s)
@@ -571,6 +573,13 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
   const int64_t tiles = (max_rows + tile_tokens - 1) / tile_tokens + f.levels;
   int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
   if (f.decode_splits > 0) splits = std::min(f.decode_splits, c->max_splits);
+  return splits;
+}
+
+int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return BALANCEKV_E_INVAL;
+  if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
+  const int splits = pick_splits(c, layer);
   {
     ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
     if (c->decode_maps)
@@ -602,6 +611,35 @@ int balancekv_decode_attn_host(balancekv_ctx* c, int layer, const void* q_host, 
 
 int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                           void* stream) {
+  // One launch when the tensor-core decode kernel serves this context and the layer's streams are
+  // in lockstep with room for the token: the kernel appends after attending (see its header).
+  if (c && layer >= 0 && layer < c->cfg.n_layers && c->decode_maps && q && out && k_new && v_new && aligned16(q) &&
+      aligned16(out) && aligned16(k_new) && aligned16(v_new)) {
+    const balancekv_config& f = c->cfg;
+    const Layout& Lo = c->Lo;
+    const std::vector<int>& streams = layer_streams(c, layer);
+    const int max_pending = Lo.T == 0 ? f.max_tokens : (f.max_pending > 0 ? std::min(f.max_pending, f.max_tokens) : f.max_tokens);
+    const StreamState& S0 = c->st[streams[0]];
+    bool fits = true;
+    for (int s : streams) {
+      const StreamState& S = c->st[s];
+      fits &= S.start0 == S0.start0 && S.len0 == S0.len0 && S.appended == S0.appended;
+      fits &= S.appended + 1 <= f.max_tokens && S.pending + 1 <= max_pending && (int64_t)S.start0 + S.len0 + 1 <= Lo.cap0;
+    }
+    if (fits) {
+      const int splits = pick_splits(c, layer);
+      const int rel = S0.start0 + S0.len0, idx0 = (int)S0.appended, new_len = S0.len0 + 1;
+      for (int s : streams) {
+        StreamState& S = c->st[s];
+        S.len0 += 1; S.appended += 1; S.pending += 1; c->tokens_appended += 1;
+      }
+      ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
+      BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
+                                      k_new, v_new, rel, idx0, new_len, static_cast<cudaStream_t>(stream)));
+      c->kernels_launched++;
+      return BALANCEKV_OK;
+    }
+  }
   int rc = balancekv_stream_append_layer(c, layer, k_new, v_new, 1, stream);
   if (rc) return rc;
   return balancekv_decode_attn(c, layer, q, out, stream);

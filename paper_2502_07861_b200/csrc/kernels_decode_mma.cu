@@ -14,6 +14,11 @@
 // tokens 16w..16w+15 of a tile and keeps a private online softmax (running max, sum, 16 x 128
 // accumulator) in registers; warps merge through shared memory, splits through a global scratch
 // and a ticket counter (the last CTA of a stream combines; nobody waits).
+// Fused decode step: with k_new / v_new given, the launch also appends one token per stream
+// (Algorithm 3's C^0 <- C^0 + {(k_j, v_j)}).  The new token never goes through the tiles: the
+// combining CTA scores it in fp32, adds it as one more partial (weight 1) and only then writes
+// its row, its position and the stream's new level-0 length, after every CTA of the stream has
+// taken its ticket, i.e. has finished reading the old segment table.
 // Rows of a tile beyond a segment's end are masked in the scores; their V rows are whatever the
 // arena holds there (zero-initialised at creation or finite older rows) times an exact zero.
 #include <cuda.h>
@@ -92,6 +97,13 @@ __device__ inline uint32_t tile_off(int token, int chunk16) {   // chunk16 in [0
   return (uint32_t)(chunk16 >> 3) * kHalf + (uint32_t)token * 128u + (uint32_t)(((chunk16 & 7) ^ (token & 7)) << 4);
 }
 
+// One appended token per stream of the layer (lockstep fill): source rows [B*H, d] and where they go.
+struct StepAppend {
+  const __nv_bfloat16* k_new;   // nullptr: plain decode
+  const __nv_bfloat16* v_new;
+  int rel_row, idx0, new_len;   // row inside the level-0 region, original position, new level-0 length
+};
+
 struct TileRef {
   int64_t row;
   int rows, level;
@@ -114,7 +126,7 @@ __device__ inline TileRef locate_tile(int tile, const int* lvl_tiles, const Seg*
 
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
-                  float* __restrict__ part, unsigned* __restrict__ tickets, int* __restrict__ status,
+                  float* __restrict__ part, unsigned* __restrict__ tickets, int* __restrict__ status, StepAppend ap,
                   const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -295,6 +307,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   float* cl = cm + 64 * kMaxGroup;                        // [splits][g] sums
   float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
   float* cL = cM + kMaxGroup;                             // [g] overall sum
+  float* cN = cL + kMaxGroup;                             // [g] factor of the appended token
   for (int i = tid; i < splits * g; i += kThreads) {
     const float* rowp = sp + (size_t)i * PS;
     cm[i] = __ldcg(rowp + kD);
@@ -308,9 +321,28 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     const float f0 = m0 == -INFINITY ? 0.f : exp2f(m0 - M), f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M);
     float L = (s0 < splits ? cl[s0 * g + h] * f0 : 0.f) + (s1 < splits ? cl[s1 * g + h] * f1 : 0.f);
     L = warp_sum(L);
-    if (s0 < splits) cm[s0 * g + h] = f0;
-    if (s1 < splits) cm[s1 * g + h] = f1;
-    if (lane == 0) { cM[h] = M; cL[h] = L; }
+    if (!ap.k_new) {
+      if (s0 < splits) cm[s0 * g + h] = f0;
+      if (s1 < splits) cm[s1 * g + h] = f1;
+    }
+    float fN = 0.f;
+    if (ap.k_new) {
+      // the appended token: level 0, weight 1; <q, k_new> in fp32, 4 dims per lane
+      const __nv_bfloat16* qh = q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane;
+      const __nv_bfloat16* kn = ap.k_new + (size_t)sl * kD + 4 * lane;
+      float dot = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dot = fmaf(__bfloat162float(qh[i]), __bfloat162float(kn[i]), dot);
+      const float x = warp_sum(dot) * sc;
+      const float M2 = fmaxf(M, x);
+      const float fS = M == -INFINITY ? 0.f : exp2f(M - M2);
+      fN = exp2f(x - M2);
+      if (s0 < splits) cm[s0 * g + h] = f0 * fS;
+      if (s1 < splits) cm[s1 * g + h] = f1 * fS;
+      if (lane == 0) { cM[h] = M2; cL[h] = fmaf(L, fS, fN); cN[h] = fN; }
+    } else if (lane == 0) {
+      cM[h] = M; cL[h] = L;
+    }
   }
   __syncthreads();
   // every thread owns 4 consecutive output columns of one head; 8 splits' loads in flight
@@ -330,10 +362,28 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
       }
     }
+    if (ap.k_new) {
+      const float fN = cN[h];
+      const __nv_bfloat16* vn = ap.v_new + (size_t)sl * kD + c;
+      acc.x = fmaf(__bfloat162float(vn[0]), fN, acc.x); acc.y = fmaf(__bfloat162float(vn[1]), fN, acc.y);
+      acc.z = fmaf(__bfloat162float(vn[2]), fN, acc.z); acc.w = fmaf(__bfloat162float(vn[3]), fN, acc.w);
+    }
     const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
     __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c);
     o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
     o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  }
+  if (ap.k_new) {
+    // append: one 256-byte row of K and of V, the position, the new length of C^0
+    const size_t dst = ((size_t)stream_base + G.region_off[0] + ap.rel_row) * kD;
+    if (tid < 16) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.K) + dst)[tid] =
+        reinterpret_cast<const uint4*>(ap.k_new + (size_t)sl * kD)[tid];
+    else if (tid < 32) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.V) + dst)[tid - 16] =
+        reinterpret_cast<const uint4*>(ap.v_new + (size_t)sl * kD)[tid - 16];
+    else if (tid == 32) {
+      A.idx[stream_base + G.region_off[0] + ap.rel_row] = ap.idx0;
+      A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
+    }
   }
   if (tid == 0) tickets[sl] = 0;   // ready for the next launch
 }
@@ -379,18 +429,32 @@ cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows
 
 void decode_mma_release(void* maps) { delete static_cast<DecodeMaps*>(maps); }
 
+cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
+                                   int splits, int* status, const void* maps, const void* k_new, const void* v_new,
+                                   int rel_row, int idx0, int new_len, cudaStream_t st);
+
 // Same scratch layout as launch_decode: ticket counters, then (stream, split, head) partial rows.
 cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                               int splits, int* status, const void* maps, cudaStream_t st) {
+  return launch_decode_step_mma(G, A, layer, q, out, scratch, splits, status, maps, nullptr, nullptr, 0, 0, 0, st);
+}
+
+// Decode attention fused with the append of one token per stream of the layer (k_new, v_new:
+// [B*H, d] bf16; all streams of the layer have the same level-0 fill).  k_new == nullptr: plain decode.
+cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
+                                   int splits, int* status, const void* maps, const void* k_new, const void* v_new,
+                                   int rel_row, int idx0, int new_len, cudaStream_t st) {
   if (!maps) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
+  const StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
+                      new_len};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q),
-                                                        static_cast<__nv_bfloat16*>(out), part, tickets, status, tm->k,
-                                                        tm->v);
+                                                        static_cast<__nv_bfloat16*>(out), part, tickets, status, ap,
+                                                        tm->k, tm->v);
   return cudaGetLastError();
 }
 
