@@ -149,7 +149,9 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     lvl_tiles[tid] = (s.len + kTN - 1) / kTN;
   }
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s <= kStages; ++s) mbar_init(&full[s], 1);       // full[kStages]: the combine's bulk copy
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -302,16 +304,38 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   __threadfence();
   // Combine: first the (max, sum) pairs of all splits in one round of loads, then every thread
   // sums its output columns over the splits with independent loads.
-  const float* sp = part + (size_t)sl * splits * g * PS;
+  const float* sp = part + (size_t)sl * splits * g * PS;   // 16-byte aligned: rows of PS * 4 = 528 bytes
   float* cm = reinterpret_cast<float*>(tiles);            // [splits][g] max, later the scale factors
   float* cl = cm + 64 * kMaxGroup;                        // [splits][g] sums
   float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
   float* cL = cM + kMaxGroup;                             // [g] overall sum
   float* cN = cL + kMaxGroup;                             // [g] factor of the appended token
+  // All partial rows of the stream are contiguous.  If they fit, one bulk copy brings them into
+  // the idle tile ring (a single round trip); otherwise they are read from global memory.
+  constexpr uint32_t kStageOff = 8192;                     // behind cm, cl, cM, cL, cN
+  const uint32_t part_bytes = (uint32_t)splits * g * PS * sizeof(float);
+  const bool staged = part_bytes <= kStages * kStageBytes - kStageOff;
+  const float* sp_s = reinterpret_cast<const float*>(tiles + kStageOff);
+  if (staged) {
+    if (tid == 0) {
+      // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
+      // (acquired above) come before the async-proxy copy
+      asm volatile("fence.proxy.async;" ::: "memory");
+      mbar_expect_tx(&full[kStages], part_bytes);
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(tiles + kStageOff)), "l"(sp), "r"(part_bytes), "r"(smem_u32(&full[kStages])) : "memory");
+    }
+    const bool landed = mbar_wait(&full[kStages], 0u);
+    if (__syncthreads_or(!landed)) {
+      if (tid == 0) { atomicCAS(status, kStatusOk, kStatusWaitTimeout); tickets[sl] = 0; }
+      return;
+    }
+    sp = sp_s;
+  }
   for (int i = tid; i < splits * g; i += kThreads) {
     const float* rowp = sp + (size_t)i * PS;
-    cm[i] = __ldcg(rowp + kD);
-    cl[i] = __ldcg(rowp + kD + 1);
+    cm[i] = staged ? rowp[kD] : __ldcg(rowp + kD);
+    cl[i] = staged ? rowp[kD + 1] : __ldcg(rowp + kD + 1);
   }
   __syncthreads();
   for (int h = warp; h < g; h += kWarps) {     // one warp per head, lanes over the (<= 64) splits
@@ -346,15 +370,17 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   }
   __syncthreads();
   // every thread owns 4 consecutive output columns of one head; 8 splits' loads in flight
-  for (int i = tid; i < g * (kD / 4); i += kThreads) {
+  const int n_items = g * (kD / 4);
+  for (int i = tid; i < n_items; i += kThreads) {
     const int h = i / (kD / 4), c = (i % (kD / 4)) * 4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < splits; s += 8) {
       float4 v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        v[u] = s + u < splits ? __ldcg(reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c))
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int u = 0; u < 8; ++u) {
+        const float4* src = reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c);
+        v[u] = s + u < splits ? (staged ? *src : __ldcg(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const float f = s + u < splits ? cm[(s + u) * g + h] : 0.f;
@@ -392,7 +418,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kStages * sizeof(uint64_t);
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (kStages + 1) * sizeof(uint64_t);
 
 }  // namespace
 
