@@ -305,7 +305,8 @@ def main():
 
     # time share of each kernel class in the timed region (sampled classes scaled to all launches)
     dc_launches = n_dec * args.steps
-    dc_total_ms = dc_ms / max(dc_n, 1) * dc_launches
+    # a launch's event bracket also holds the gap to its neighbours, so the loop time bounds the total
+    dc_total_ms = min(dc_ms / max(dc_n, 1) * dc_launches, float(t_dec.sum()))
     kernels = dict(
         gram_walk=dict(bound="tensor", achieved=tensor_ach, peak=peaks["tensor"], unit="TFLOP/s",
                        frac=tensor_ach / peaks["tensor"], traffic=None, ms_per_launch=gw_ms_per_launch, launches=gw_n,

@@ -121,7 +121,10 @@ int balancekv_decode_attn(balancekv_ctx* ctx, int layer, const void* q, void* ou
  * balancekv_stream_append_layer(.., 1) followed by balancekv_decode_attn. */
 int balancekv_stream_step(balancekv_ctx* ctx, int layer, const void* q, const void* k_new, const void* v_new,
                           void* out, void* stream);
-/* Same with HOST buffers for q, k_new, v_new and out (see the other *_host calls). */
+/* Same with HOST buffers for q, k_new, v_new and out.  The inputs are read by the CPU during
+ * the call (packed into a pinned staging slot of the context and sent as one transfer), so the
+ * caller may reuse them as soon as the call returns; out_host is written in stream order
+ * (synchronise the stream before reading it).  The first call allocates the staging buffers. */
 int balancekv_stream_step_host(balancekv_ctx* ctx, int layer, const void* q_host, const void* k_host,
                                const void* v_host, void* out_host, void* stream);
 

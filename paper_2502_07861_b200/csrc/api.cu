@@ -90,6 +90,14 @@ struct balancekv_ctx {
   size_t bounce_bytes = 0;
   void* bounce_q = nullptr;
   void* bounce_out = nullptr;
+  // stream_step_host: q | k_new | v_new of a step packed into one pinned slot, one copy to the device
+  static constexpr int kStepSlots = 64;
+  char* step_host = nullptr;            // pinned, kStepSlots slots
+  char* step_dev_in = nullptr;          // q | k | v
+  void* step_dev_out = nullptr;
+  size_t step_slot_bytes = 0;
+  cudaEvent_t step_ev[kStepSlots] = {};
+  unsigned long long step_count = 0;
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
   std::vector<std::vector<int>> layer_stream_ids;
@@ -325,10 +333,13 @@ int balancekv_destroy(balancekv_ctx* c) {
   decode_mma_release(c->decode_maps);
   void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
                   c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
-                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out};
+                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->h_ring) cudaFreeHost(c->h_ring);
+  if (c->step_host) cudaFreeHost(c->step_host);
+  for (cudaEvent_t e : c->step_ev)
+    if (e) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i)
     if (c->ring_ev[i]) cudaEventDestroy(c->ring_ev[i]);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
@@ -647,9 +658,35 @@ int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void
 
 int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, const void* k_host, const void* v_host,
                                void* out_host, void* stream) {
-  int rc = balancekv_stream_append_layer_host(c, layer, k_host, v_host, 1, stream);
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !q_host || !k_host || !v_host || !out_host) return BALANCEKV_E_INVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t qb = (size_t)c->cfg.n_seqs * c->cfg.n_q_heads * c->cfg.head_dim * c->esz;
+  const size_t kb = (size_t)c->cfg.n_seqs * c->cfg.n_kv_heads * c->cfg.head_dim * c->esz;
+  if (!c->step_host) {   // first call: staging buffers (allocates)
+    c->step_slot_bytes = (qb + 2 * kb + 255) / 256 * 256;
+    BKV_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->step_host), c->step_slot_bytes * balancekv_ctx::kStepSlots,
+                           cudaHostAllocDefault));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->step_dev_in), c->step_slot_bytes));
+    BKV_CUDA(cudaMalloc(&c->step_dev_out, qb));
+    c->bytes_resident += c->step_slot_bytes + qb;
+    for (cudaEvent_t& e : c->step_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
+  // The three small inputs travel as one copy: packed into a pinned slot on the host (a slot is
+  // reused only after the copy that read it has finished), then one host-to-device transfer.
+  const int slot = (int)(c->step_count % balancekv_ctx::kStepSlots);
+  if (c->step_count >= (unsigned long long)balancekv_ctx::kStepSlots) BKV_CUDA(cudaEventSynchronize(c->step_ev[slot]));
+  ++c->step_count;
+  char* h = c->step_host + (size_t)slot * c->step_slot_bytes;
+  std::memcpy(h, q_host, qb);
+  std::memcpy(h + qb, k_host, kb);
+  std::memcpy(h + qb + kb, v_host, kb);
+  BKV_CUDA(cudaMemcpyAsync(c->step_dev_in, h, qb + 2 * kb, cudaMemcpyHostToDevice, st));
+  BKV_CUDA(cudaEventRecord(c->step_ev[slot], st));
+  int rc = balancekv_stream_step(c, layer, c->step_dev_in, c->step_dev_in + qb, c->step_dev_in + qb + kb, c->step_dev_out,
+                                 stream);
   if (rc) return rc;
-  return balancekv_decode_attn_host(c, layer, q_host, out_host, stream);
+  BKV_CUDA(cudaMemcpyAsync(out_host, c->step_dev_out, qb, cudaMemcpyDeviceToHost, st));
+  return BALANCEKV_OK;
 }
 
 int balancekv_level_sizes(balancekv_ctx* c, int seq, int layer, int kv_head, int32_t* sizes) {

@@ -130,3 +130,36 @@ def test_profiler_class_mask_and_sampling(cuda_lib):
     ctx.profile_enable(False)
     ctx.decode_attn(0, q)
     assert ctx.profile_read()["decode"][0] == 0
+
+
+def test_host_buffer_entry_points_match_the_device_ones(cuda_lib):
+    """append / decode / step through pinned host buffers (more steps than staging slots) give
+    bit-identical caches and outputs to the device-pointer calls."""
+    Bs, Hs, g, d, n, steps = 2, 2, 4, 128, 200, 70
+    mk = lambda: cuda_lib.Context(n_seqs=Bs, n_layers=1, n_kv_heads=Hs, n_q_heads=Hs * g, head_dim=d, dtype="bf16",
+                                  block=64, levels=1, max_tokens=n + steps, seed=1)
+    rng = np.random.default_rng(1)
+    bf = lambda shape: torch.from_numpy(rng.standard_normal(shape).astype(np.float32)).to(torch.bfloat16)
+    K_h, V_h = bf((Bs, Hs, n, d)).pin_memory(), bf((Bs, Hs, n, d)).pin_memory()
+    a, b = mk(), mk()
+    a.stream_append_layer(0, K_h.cuda(), V_h.cuda())
+    b.stream_append_layer_host(0, K_h, V_h)
+    a.compress()
+    b.compress()
+    q_h = bf((Bs, Hs * g, d)).pin_memory()
+    out_h = torch.empty_like(q_h).pin_memory()
+    b.decode_attn_host(0, q_h, out_h)
+    torch.cuda.synchronize()
+    assert torch.equal(a.decode_attn(0, q_h.cuda()).cpu(), out_h)
+    qs, ks, vs = bf((steps, Bs, Hs * g, d)).pin_memory(), bf((steps, Bs, Hs, 1, d)).pin_memory(), bf((steps, Bs, Hs, 1, d)).pin_memory()
+    outs_h = torch.empty_like(qs).pin_memory()
+    out_d = torch.empty(Bs, Hs * g, d, dtype=torch.bfloat16, device="cuda")
+    for s in range(steps):
+        b.stream_step_host(0, qs[s], ks[s], vs[s], outs_h[s])
+    for s in range(steps):
+        a.stream_step(0, qs[s].cuda(), ks[s].cuda(), vs[s].cuda(), out_d)
+        if s in (0, steps // 2, steps - 1):
+            torch.cuda.synchronize()
+            assert torch.equal(out_d.cpu(), outs_h[s])
+    for h in range(Hs):
+        assert all(torch.equal(x, y) for x, y in zip(a.cache_view(1, 0, h), b.cache_view(1, 0, h)))
