@@ -307,14 +307,18 @@ def main():
     dc_launches = n_dec * args.steps
     # a launch's event bracket also holds the gap to its neighbours, so the loop time bounds the total
     dc_total_ms = min(dc_ms / max(dc_n, 1) * dc_launches, float(t_dec.sum()))
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+    # summarised under profiles/ (average of the level-0 and level-1 launches; the decode figure is
+    # a cold-L2 launch of the same shape, while this loop re-reads its cache from L2)
+    traffic = dict(gram_walk=103.0e6, compact=64.2e6, decode=33.65e6) if (n_ctx, t, T, B * H) == (32768, 1024, 2, 8) else {}
     kernels = dict(
         gram_walk=dict(bound="tensor", achieved=tensor_ach, peak=peaks["tensor"], unit="TFLOP/s",
-                       frac=tensor_ach / peaks["tensor"], traffic=None, ms_per_launch=gw_ms_per_launch, launches=gw_n,
+                       frac=tensor_ach / peaks["tensor"], traffic=traffic.get("gram_walk"), ms_per_launch=gw_ms_per_launch, launches=gw_n,
                        ms_total=gw_ms),
         compact=dict(bound="hbm", achieved=cp_gbs, peak=peaks["hbm"], unit="GB/s", frac=cp_gbs / peaks["hbm"],
-                     traffic=None, ms_per_launch=cp_ms / max(cp_n, 1), launches=cp_n, ms_total=cp_ms),
+                     traffic=traffic.get("compact"), ms_per_launch=cp_ms / max(cp_n, 1), launches=cp_n, ms_total=cp_ms),
         decode=dict(bound="hbm", achieved=dc_gbs, peak=peaks["hbm"], unit="GB/s", frac=dc_gbs / peaks["hbm"],
-                    traffic=None, ms_per_launch=dc_ms / max(dc_n, 1), launches=dc_launches, launches_timed=dc_n,
+                    traffic=traffic.get("decode"), ms_per_launch=dc_ms / max(dc_n, 1), launches=dc_launches, launches_timed=dc_n,
                     ms_total=dc_total_ms,
                     note="the cache of this workload (35 MB) stays in L2 between decode steps; HBM-bound shapes are "
                          "timed by `python -m paper_2502_07861_b200.microbench decode`"))
