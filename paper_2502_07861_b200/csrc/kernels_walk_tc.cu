@@ -221,7 +221,8 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   const int t = G.t, P = t / kTile;
   float* etas = reinterpret_cast<float*>(sm + Smem::kTilesEnd);          // [t] signs scaled by 1/r_value^2 (0 = undecided)
   float* xs = etas + t;                                                   // [3][128] partial correlations of column quarters 1..3
-  float* thr_s = xs + (kEpiGroups - 1) * kTile;                           // [t] decision thresholds c (1 - 2 u_j)
+  float* xb = xs + (kEpiGroups - 1) * kTile;                              // [3][128] ... and of their sums of |Ghat|
+  float* thr_s = xb + (kEpiGroups - 1) * kTile;                           // [t] decision thresholds c (1 - 2 u_j)
   int8_t* eta8 = reinterpret_cast<int8_t*>(thr_s + t);                    // [t] signs
   uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
   // x = 0: the K K^T product, x = 1: the V V^T product
@@ -454,6 +455,15 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       // The walk over the panel's 128 tokens by sweeps: group 0 owns the decisions, groups 1-3
       // supply the partial sums of their columns.  Undecided signs are stored as 0.
       const float4* e4 = reinterpret_cast<const float4*>(etas + r * kTile + col0);
+      // In sweep 0 (all in-panel signs still 0, S = the earlier panels' part) a row whose distance
+      // to its threshold exceeds sum_j |Ghat_ij| of its in-panel columns is already decided; if
+      // that holds for every row (and no row can FAIL, and S is not recorded) one sweep suffices.
+      float absum = 0.f;
+      if (below) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) absum += fabsf(g[i]);
+      }
+      if (wg > 0) xb[(wg - 1) * kTile + row] = absum;
       bool plus = false;
       float S = 0.f;
 #pragma unroll 1
@@ -477,7 +487,13 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
           bar_sync(1, kEpiThreads);                       // all partial sums of this sweep are written
           S = (part + xs[row]) + (xs[kTile + row] + xs[2 * kTile + row]);
           const bool now = S < thr;
-          changed = sweep == 0 || now != plus;
+          if (sweep == 0) {
+            const float bound = ((absum + xb[row]) + (xb[kTile + row] + xb[2 * kTile + row])) * inv_rv2;
+            const float slack = 1e-5f * (fabsf(S) + bound) + 1e-30f;
+            changed = C.dbg_off >= 0 || !(fabsf(S - thr) > bound + slack) || !(fabsf(S) + bound + slack < cw);
+          } else {
+            changed = now != plus;
+          }
           plus = now;
           etas[j] = plus ? inv_rv2 : -inv_rv2;
         }
@@ -513,7 +529,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 9 + (kEpiGroups - 1) * kTile * 4 + 256; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 9 + 2 * (kEpiGroups - 1) * kTile * 4 + 256; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
