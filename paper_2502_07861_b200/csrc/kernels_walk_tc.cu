@@ -23,6 +23,8 @@
 // its rows in slot r % 3 and streams its column tiles through the other two, and the rows of
 // panel r + 1 are fetched into the slot that panel r's column tiles leave first, so the next
 // panel's first products are already in TMEM when the walk of the diagonal tile ends.
+// Inside a slot every operand is two boxes of 64 dims with their own full/empty barriers: a box is
+// refilled as soon as the four MMAs that read it have retired.
 // Ghat never touches global memory.
 //
 // Every wait is bounded: a wait that runs out sets the abort flag and the status word, all
@@ -132,13 +134,16 @@ __device__ inline void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) 
       "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "n"(kAccumulate), "r"(kInstrDesc) : "memory");
 }
-// The 8 K-steps of one 128 x 128 x 128 product: A and B tiles given by their descriptor low words.
-__device__ inline void umma_tile(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
-  constexpr uint32_t kHalf = kHalfBytes >> 4;
+// The 8 K-steps of one 128 x 128 x 128 product in two halves (dims 0..63, then 64..127, which sit
+// kHalfBytes further): A and B tiles given by their descriptor low words.
+__device__ inline void umma_tile_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
   umma_bf16<0>(d_tmem, a_lo, b_lo);
   umma_bf16<1>(d_tmem, a_lo + 2, b_lo + 2);
   umma_bf16<1>(d_tmem, a_lo + 4, b_lo + 4);
   umma_bf16<1>(d_tmem, a_lo + 6, b_lo + 6);
+}
+__device__ inline void umma_tile_hi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo) {
+  constexpr uint32_t kHalf = kHalfBytes >> 4;
   umma_bf16<1>(d_tmem, a_lo + kHalf, b_lo + kHalf);
   umma_bf16<1>(d_tmem, a_lo + kHalf + 2, b_lo + kHalf + 2);
   umma_bf16<1>(d_tmem, a_lo + kHalf + 4, b_lo + kHalf + 4);
@@ -226,11 +231,13 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   int8_t* eta8 = reinterpret_cast<int8_t*>(thr_s + t);                    // [t] signs
   uint64_t* bars = reinterpret_cast<uint64_t*>(eta8 + t);                 // t is a multiple of 128
   // x = 0: the K K^T product, x = 1: the V V^T product
-  uint64_t* full = bars + 0;         // [x][3] operand tile of product x landed in slot s
-  uint64_t* empty = bars + 6;        // [x][3] product x no longer reads slot s -> producer
-  uint64_t* xdone = bars + 12;       // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
-  uint64_t* tmem_empty = bars + 16;  // [2] both warpgroups have drained buffer b
-  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 18);
+  // An operand tile travels as two boxes of 64 dims (h = 0, 1); a box is refilled as soon as the
+  // four MMAs that read it are done, which lengthens the prefetch distance of the column ring.
+  uint64_t* full = bars + 0;         // [x][3][h] box h of product x's operand landed in slot s: index 6 x + 2 s + h
+  uint64_t* empty = bars + 12;       // [x][3][h] product x no longer reads that box -> producer
+  uint64_t* xdone = bars + 24;       // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
+  uint64_t* tmem_empty = bars + 28;  // [2] all epilogue warps have drained buffer b
+  uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 30);
   int* abort_flag = reinterpret_cast<int*>(tmem_ptr_s + 1);
 
   const int call = blockIdx.x;
@@ -238,7 +245,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
-    for (int i = 0; i < 6; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); }
+    for (int i = 0; i < 12; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); }
     for (int i = 0; i < 4; ++i) mbar_init(xdone + i, 1);
     for (int i = 0; i < 2; ++i) mbar_init(tmem_empty + i, kEpiWarps);       // one arrival per warp (lane 0 after __syncwarp)
     *abort_flag = 0;
@@ -274,14 +281,17 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
         if (again) par ^= 1u << slot;
         unsigned char* st = sm + (uint32_t)slot * Smem::kSlotBytes;
         const int y = (int)(C.src_row + (int64_t)tile_row * kTile);
-        if (again && !wait_bar(empty + slot, ph, abort_flag)) return false;
-        mbar_expect_tx(full + slot, kTileBytes);
-        tma_load_2d(st, &tmK, 0, y, full + slot);
-        tma_load_2d(st + kHalfBytes, &tmK, 64, y, full + slot);
-        if (again && !wait_bar(empty + 3 + slot, ph, abort_flag)) return false;
-        mbar_expect_tx(full + 3 + slot, kTileBytes);
-        tma_load_2d(st + kTileBytes, &tmV, 0, y, full + 3 + slot);
-        tma_load_2d(st + kTileBytes + kHalfBytes, &tmV, 64, y, full + 3 + slot);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint64_t* fk = full + 2 * slot + h;
+          uint64_t* fv = full + 6 + 2 * slot + h;
+          if (again && !wait_bar(empty + 2 * slot + h, ph, abort_flag)) return false;
+          mbar_expect_tx(fk, kHalfBytes);
+          tma_load_2d(st + h * kHalfBytes, &tmK, 64 * h, y, fk);
+          if (again && !wait_bar(empty + 6 + 2 * slot + h, ph, abort_flag)) return false;
+          mbar_expect_tx(fv, kHalfBytes);
+          tma_load_2d(st + kTileBytes + h * kHalfBytes, &tmV, 64 * h, y, fv);
+        }
         return true;
       };
       ok = load(0, 0);
@@ -302,23 +312,27 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       constexpr uint32_t kSlotDesc = Smem::kSlotBytes >> 4;
       for (int r = 0; r < P && ok; ++r) {
         const int rs = r % 3;
-        if (!(ok = wait_bar(full + 3 * x + rs, (par >> rs) & 1u, abort_flag))) break;
+        if (!(ok = wait_bar(full + 6 * x + 2 * rs, (par >> rs) & 1u, abort_flag))) break;
+        if (!(ok = wait_bar(full + 6 * x + 2 * rs + 1, (par >> rs) & 1u, abort_flag))) break;
         par ^= 1u << rs;
         const uint32_t arow = slot0 + (uint32_t)rs * kSlotDesc;
         for (int c = 0; c <= r; ++c, ++i) {
           const int buf = i & 1;
           if (!(ok = wait_bar(tmem_empty + buf, (uint32_t)(((i >> 1) & 1) ^ 1), abort_flag))) break;
-          uint32_t b = arow;
-          int slot = rs;
+          const int slot = c < r ? (r + 1 + (c & 1)) % 3 : rs;
+          const uint32_t b = slot0 + (uint32_t)slot * kSlotDesc;
+          const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256u + (x ? 128u : 0u);
+          const uint32_t ph = (par >> slot) & 1u;
           if (c < r) {
-            slot = (r + 1 + (c & 1)) % 3;
-            if (!(ok = wait_bar(full + 3 * x + slot, (par >> slot) & 1u, abort_flag))) break;
+            if (!(ok = wait_bar(full + 6 * x + 2 * slot, ph, abort_flag))) break;
             par ^= 1u << slot;
-            b = slot0 + (uint32_t)slot * kSlotDesc;
           }
           tc_fence_after();
-          umma_tile(tmem_base + (uint32_t)buf * 256u + (x ? 128u : 0u), arow, b);
-          umma_commit(empty + 3 * x + slot);     // a column slot after its tile, the row slot after the diagonal tile
+          umma_tile_lo(d_tmem, arow, b);
+          umma_commit(empty + 6 * x + 2 * slot);       // a column slot's box after its tile, the row slot's after the diagonal tile
+          if (c < r && !(ok = wait_bar(full + 6 * x + 2 * slot + 1, ph, abort_flag))) break;
+          umma_tile_hi(d_tmem, arow, b);
+          umma_commit(empty + 6 * x + 2 * slot + 1);
           umma_commit(xdone + 2 * x + buf);
         }
       }
