@@ -11,7 +11,9 @@ from .binding import (  # noqa: F401
     num_threads,
     philox4x32_10,
     softmax_balance,
+    two_instance_estimate,
     walk_constant,
     walk_uniform,
     weighted_attention,
+    weighted_sums,
 )

@@ -8,7 +8,8 @@
 //   * the strict n/2 selection of the "Implementation Detail" paragraph of Appendix B,
 //   * MergeAndReduce (Algorithm 3) with its estimator (Theorem 3.3),
 //   * the attention definition Eq. (1) and the weighted estimator ratio of
-//     Algorithm 1's output ratio, evaluated over one shared weighted set.
+//     Algorithm 1's output ratio, evaluated over one shared weighted set, and its two
+//     un-normalised halves for the form with a separate denominator instance.
 //
 // It shares no code with the CUDA library: no common header, helper, table or
 // constant generator.  Only tests, the smoke check and the bench's cpu_baseline /
@@ -17,7 +18,8 @@
 //
 // Parity pins (see tests/test_oracle_*.py): Philox known-answer vectors; T=0 equals
 // Eq. (1); weight-sum and level-size invariants; brute-force enumeration of the walk
-// law for m<=16; closed forms of the kernel; the Theorem 3.2 bound with explicit c.
+// law for m<=16; closed forms of the kernel; the Theorem 3.2 bound with explicit c; the
+// un-normalised sums against a direct evaluation and against the pinned ratio.
 //
 // Build: g++ -O2 -fopenmp -shared -fPIC balancekv_oracle.cpp -o libbalancekv_oracle.so
 
@@ -407,6 +409,30 @@ void okv_stream_exact(void* h, const double* q, int nq, double* out) {
   for (int a = 0; a < nq; ++a)
     weighted_attention(s->K.data(), s->V.data(), nullptr, s->n, s->P.d, q + (size_t)a * s->P.d,
                        out + (size_t)a * s->P.d);
+}
+
+// Un-normalised weighted sums over explicit arrays (the two halves of Algorithm 1's output ratio,
+// which takes its numerator from the sets V^l of one MergeAndReduce instance and its denominator
+// from the sets K^l of another):  with m = max_i (<k_i,q>/sqrt d + ln w_i),
+//   num[c] = sum_i w_i e^{<k_i,q>/sqrt d - m} v_i[c],   den = sum_i w_i e^{<k_i,q>/sqrt d - m},   logmax = m.
+void okv_weighted_sums(const double* K, const double* V, const double* w, int64_t len, int d, const double* q,
+                       int nq, double* num, double* den, double* logmax) {
+  const double inv_sqrt_d = 1.0 / std::sqrt((double)d);
+  for (int a = 0; a < nq; ++a) {
+    const double* qa = q + (size_t)a * d;
+    double mx = -INFINITY;
+    for (int64_t i = 0; i < len; ++i)
+      mx = std::max(mx, dot(K + i * d, qa, d) * inv_sqrt_d + std::log(w ? w[i] : 1.0));
+    double Z = 0.0;
+    for (int c = 0; c < d; ++c) num[(size_t)a * d + c] = 0.0;
+    for (int64_t i = 0; i < len; ++i) {
+      const double e = std::exp(dot(K + i * d, qa, d) * inv_sqrt_d + std::log(w ? w[i] : 1.0) - mx);
+      Z += e;
+      for (int c = 0; c < d; ++c) num[(size_t)a * d + c] += e * V[i * d + c];
+    }
+    den[a] = Z;
+    logmax[a] = mx;
+  }
 }
 
 // Weighted attention over explicit arrays: K,V [len,d], w [len] (null = all ones).

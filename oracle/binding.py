@@ -94,6 +94,8 @@ def _load():
     lib.okv_stream_exact.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
     lib.okv_weighted_attn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
                                       C.c_void_p, C.c_int, C.c_void_p]
+    lib.okv_weighted_sums.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int,
+                                      C.c_void_p, C.c_void_p, C.c_void_p]
     lib.okv_num_threads.restype = C.c_int
     _ = dp
     _lib = lib
@@ -156,6 +158,30 @@ def weighted_attention(K, V, w, q):
     _load().okv_weighted_attn(_ptr(K), _ptr(V), _ptr(wv), K.shape[0], K.shape[1], _ptr(q),
                               q.shape[0], _ptr(out))
     return out
+
+
+def weighted_sums(K, V, w, q):
+    """(num [nq,d], den [nq], logmax [nq]): sum w e^{<k,q>/sqrt d - m} v, sum w e^{... - m}, m (natural log)."""
+    K = _f64(K)
+    V = _f64(V)
+    q = _f64(q).reshape(-1, K.shape[1])
+    wv = None if w is None else _f64(w)
+    num = np.zeros_like(q)
+    den = np.zeros(q.shape[0])
+    mx = np.zeros(q.shape[0])
+    _load().okv_weighted_sums(_ptr(K), _ptr(V), _ptr(wv), K.shape[0], K.shape[1], _ptr(q), q.shape[0],
+                              _ptr(num), _ptr(den), _ptr(mx))
+    return num, den, mx
+
+
+def two_instance_estimate(numerator_view, denominator_view, q):
+    """Algorithm 1's output ratio from the (K, V, w) view of the numerator instance and the
+    (K, ., w) view of the denominator instance."""
+    Kn, Vn, wn = numerator_view[:3]
+    Kd, Vd, wd = denominator_view[:3]
+    num, _, mn = weighted_sums(Kn, Vn, wn, q)
+    _, den, md = weighted_sums(Kd, Vd, wd, q)
+    return num * np.exp(mn - md)[:, None] / den[:, None]
 
 
 class OracleStream:
