@@ -189,6 +189,22 @@ int balancekv_debug_call(balancekv_ctx* ctx, int seq, int layer, int kv_head, in
  * configuration and debug buffers are kept.  Enqueued on `stream`. */
 int balancekv_reset(balancekv_ctx* ctx, void* stream);
 
+/* Algorithm 1 with its separate denominator instance (MR-Denominator), without the value-norm
+ * buckets.  The caller dedicates two layer slots of the context to one model layer: slot
+ * `layer_num` receives (k_j, v_j) through the ordinary append calls, slot `layer_den` receives
+ * (k_j, 1) through balancekv_stream_append_layer_keys (K: [n_seqs, n_kv_heads, n_tokens, head_dim]
+ * device; the library supplies the unit value (1, 0, ..., 0), for which the pairwise kernel of
+ * Algorithm 2 becomes exp(<k_i, k_j>/sqrt d)).  balancekv_compress then runs MergeAndReduce on
+ * both, with independent coins (the coin's counter holds the slot index), and
+ *   balancekv_decode_attn_two:  out = sum_l 2^l sum_{V^l} e^{<k,q>/sqrt d} v
+ *                                   / sum_l 2^l sum_{K^l} e^{<k,q>/sqrt d}
+ * (Algorithm 1's output ratio), V^l the sets of slot layer_num and K^l those of slot layer_den.
+ * bf16, head_dim 128, group <= 8 only (else BALANCEKV_E_INVAL); q, out as balancekv_decode_attn.
+ * The first call of either function allocates its buffers. */
+int balancekv_stream_append_layer_keys(balancekv_ctx* ctx, int layer, const void* K, int n_tokens, void* stream);
+int balancekv_decode_attn_two(balancekv_ctx* ctx, int layer_num, int layer_den, const void* q, void* out,
+                              void* stream);
+
 /* Kernel timing for roofline reports.  While enabled, every launch of the kernel classes
  * below is bracketed by CUDA events on its launch stream (at most 8192 launches between two
  * reads; later ones are not recorded).  balancekv_profile_read synchronises the device and

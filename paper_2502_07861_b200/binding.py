@@ -22,7 +22,8 @@ EXPORTS = [
     "balancekv_cache_view", "balancekv_level_sizes", "balancekv_debug_enable", "balancekv_debug_call",
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
-    "balancekv_stream_step", "balancekv_stream_step_host",
+    "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
+    "balancekv_decode_attn_two",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -86,6 +87,8 @@ def load():
     lib.balancekv_stream_step_host.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.balancekv_profile_enable.argtypes = [vp, ci]
     lib.balancekv_profile_sample.argtypes = [vp, ci, ci]
+    lib.balancekv_stream_append_layer_keys.argtypes = [vp, ci, vp, ci, vp]
+    lib.balancekv_decode_attn_two.argtypes = [vp, ci, ci, vp, vp, vp]
     lib.balancekv_profile_read.argtypes = [vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     for name in EXPORTS:
@@ -210,6 +213,21 @@ class Context:
         _check(self.lib.balancekv_stream_step(self._h, layer, self._dev(q, "q"), self._dev(k_new, "k_new"),
                                               self._dev(v_new, "v_new"), self._dev(out, "out"), _stream_ptr(stream)),
                "balancekv_stream_step")
+        return out
+
+    def stream_append_layer_keys(self, layer, K, stream=None):
+        """Denominator instance of Algorithm 1: append (k_j, 1); K [B, H, n, d] on the device."""
+        _check(self.lib.balancekv_stream_append_layer_keys(self._h, layer, self._dev(K, "K"), K.shape[2],
+                                                           _stream_ptr(stream)), "balancekv_stream_append_layer_keys")
+
+    def decode_attn_two(self, layer_num, layer_den, q, out=None, stream=None):
+        """Algorithm 1's output ratio: numerator from slot layer_num, denominator from slot layer_den."""
+        import torch
+
+        if out is None:
+            out = torch.empty_like(q)
+        _check(self.lib.balancekv_decode_attn_two(self._h, layer_num, layer_den, self._dev(q, "q"), self._dev(out, "out"),
+                                                  _stream_ptr(stream)), "balancekv_decode_attn_two")
         return out
 
     def stream_step_host(self, layer, q_host, k_host, v_host, out_host, stream=None):

@@ -20,6 +20,10 @@ void walk_tc_release(void* tmaps);
 bool decode_mma_supported(const Geom& G);
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out);
 void decode_mma_release(void* maps);
+cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
+                                    float* scratch, int splits, int* status, const void* maps, cudaStream_t st);
+cudaError_t launch_two_instance_ratio(const float* acc_n, const float* ml_n, const float* ml_d, void* out, int n_heads, int d,
+                                      cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
                                    int rel_row, int idx0, int new_len, cudaStream_t st);
@@ -98,6 +102,11 @@ struct balancekv_ctx {
   size_t step_slot_bytes = 0;
   cudaEvent_t step_ev[kStepSlots] = {};
   unsigned long long step_count = 0;
+  // two-instance estimator: un-normalised parts of the numerator and denominator instances, unit values
+  float* two_acc = nullptr;             // [B, Hq, d] numerator sums
+  float* two_ml = nullptr;              // [2][B, Hq, 2] (max, sum) of the numerator and of the denominator instance
+  void* unit_V = nullptr;               // rows (1, 0, ..., 0) for balancekv_stream_append_layer_keys
+  size_t unit_rows = 0;
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
   std::vector<std::vector<int>> layer_stream_ids;
@@ -333,7 +342,7 @@ int balancekv_destroy(balancekv_ctx* c) {
   decode_mma_release(c->decode_maps);
   void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
                   c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
-                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out};
+                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->unit_V};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->h_ring) cudaFreeHost(c->h_ring);
@@ -617,6 +626,62 @@ int balancekv_decode_attn_host(balancekv_ctx* c, int layer, const void* q_host, 
   int rc = balancekv_decode_attn(c, layer, c->bounce_q, c->bounce_out, stream);
   if (rc) return rc;
   BKV_CUDA(cudaMemcpyAsync(out_host, c->bounce_out, bytes, cudaMemcpyDeviceToHost, st));
+  return BALANCEKV_OK;
+}
+
+int balancekv_stream_append_layer_keys(balancekv_ctx* c, int layer, const void* K, int n_tokens, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !K || n_tokens < 0) return BALANCEKV_E_INVAL;
+  if (n_tokens == 0) return BALANCEKV_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t rows = (size_t)c->cfg.n_seqs * c->cfg.n_kv_heads * n_tokens;
+  if (rows > c->unit_rows) {   // (re)build the unit-value rows: the value "1" of Algorithm 1's denominator instance
+    const size_t rb = (size_t)c->cfg.head_dim * c->esz;
+    BKV_CUDA(cudaStreamSynchronize(st));
+    if (c->unit_V) { cudaFree(c->unit_V); c->bytes_resident -= c->unit_rows * rb; }
+    c->unit_V = nullptr; c->unit_rows = 0;
+    BKV_CUDA(cudaMalloc(&c->unit_V, rows * rb));
+    BKV_CUDA(cudaMemsetAsync(c->unit_V, 0, rows * rb, st));
+    // element 0 of every row = 1.0 (bf16 0x3F80 / fp32 0x3F800000): a strided 2-D set of the high bytes
+    if (c->esz == 2) {
+      BKV_CUDA(cudaMemset2DAsync(static_cast<char*>(c->unit_V) + 1, rb, 0x3F, 1, rows, st));
+      BKV_CUDA(cudaMemset2DAsync(c->unit_V, rb, 0x80, 1, rows, st));
+    } else {
+      BKV_CUDA(cudaMemset2DAsync(static_cast<char*>(c->unit_V) + 3, rb, 0x3F, 1, rows, st));
+      BKV_CUDA(cudaMemset2DAsync(static_cast<char*>(c->unit_V) + 2, rb, 0x80, 1, rows, st));
+    }
+    c->unit_rows = rows; c->bytes_resident += rows * rb;
+  }
+  return append_impl(c, layer_streams(c, layer), 0, K, c->unit_V, nullptr, n_tokens, st, layer);
+}
+
+int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, const void* q, void* out, void* stream) {
+  if (!c || !q || !out || layer_num < 0 || layer_num >= c->cfg.n_layers || layer_den < 0 || layer_den >= c->cfg.n_layers)
+    return BALANCEKV_E_INVAL;
+  if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
+  if (!c->decode_maps) return BALANCEKV_E_INVAL;          // bf16, head_dim 128, group <= 8 only
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_heads = c->cfg.n_seqs * c->cfg.n_q_heads, d = c->cfg.head_dim;
+  if (!c->two_acc) {   // first call: buffers for the un-normalised parts (allocates)
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_acc), sizeof(float) * (size_t)n_heads * d * 2));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_ml), sizeof(float) * (size_t)n_heads * 4));
+    c->bytes_resident += sizeof(float) * ((size_t)n_heads * d * 2 + (size_t)n_heads * 4);
+  }
+  float* acc_n = c->two_acc;
+  float* acc_d = c->two_acc + (size_t)n_heads * d;        // the denominator instance's value sums are not used
+  float* ml_n = c->two_ml;
+  float* ml_d = c->two_ml + (size_t)n_heads * 2;
+  {
+    ProfScope ps(c, 4, st);
+    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_num, q, acc_n, ml_n, c->d_decode_scratch, pick_splits(c, layer_num),
+                                     c->d_status, c->decode_maps, st));
+  }
+  {
+    ProfScope ps(c, 4, st);
+    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_den, q, acc_d, ml_d, c->d_decode_scratch, pick_splits(c, layer_den),
+                                     c->d_status, c->decode_maps, st));
+  }
+  BKV_CUDA(launch_two_instance_ratio(acc_n, ml_n, ml_d, out, n_heads, d, st));
+  c->kernels_launched += 3;
   return BALANCEKV_OK;
 }
 

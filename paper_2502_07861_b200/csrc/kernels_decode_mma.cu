@@ -102,6 +102,12 @@ struct StepAppend {
   const __nv_bfloat16* k_new;   // nullptr: plain decode
   const __nv_bfloat16* v_new;
   int rel_row, idx0, new_len;   // row inside the level-0 region, original position, new level-0 length
+  // Un-normalised result instead of the ratio (both nullptr: ratio in `out`): per query head
+  // sum_i w_i e^{l_i - M} v_i as fp32 [B, H g, d] and (M, sum_i w_i e^{l_i - M}) as fp32 [B, H g, 2],
+  // M the largest base-2 logit incl. log2 w_i.  Algorithm 1 divides the numerator of one
+  // MergeAndReduce instance by the denominator of another; this is one such part.
+  float* raw_acc;
+  float* raw_ml;
 };
 
 struct TileRef {
@@ -394,6 +400,12 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       acc.x = fmaf(__bfloat162float(vn[0]), fN, acc.x); acc.y = fmaf(__bfloat162float(vn[1]), fN, acc.y);
       acc.z = fmaf(__bfloat162float(vn[2]), fN, acc.z); acc.w = fmaf(__bfloat162float(vn[3]), fN, acc.w);
     }
+    if (ap.raw_acc) {
+      const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
+      *reinterpret_cast<float4*>(ap.raw_acc + qh * kD + c) = acc;
+      if (c == 0) { ap.raw_ml[2 * qh] = cM[h]; ap.raw_ml[2 * qh + 1] = cL[h]; }
+      continue;
+    }
     const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
     __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c);
     o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
@@ -465,6 +477,41 @@ cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const vo
   return launch_decode_step_mma(G, A, layer, q, out, scratch, splits, status, maps, nullptr, nullptr, 0, 0, 0, st);
 }
 
+// Un-normalised parts (see StepAppend::raw_acc) of the layer's streams for the two-instance estimator.
+cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
+                                    float* scratch, int splits, int* status, const void* maps, cudaStream_t st) {
+  if (!maps || !raw_acc || !raw_ml) return cudaErrorInvalidValue;
+  const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
+  const int n_sl = G.B * G.H;
+  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
+  float* part = scratch + ((n_sl + 63) / 64) * 64;
+  dim3 grid(n_sl, splits);
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml};
+  decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
+                                                        tickets, status, ap, tm->k, tm->v);
+  return cudaGetLastError();
+}
+
+// out = numerator parts / denominator parts: z = acc_n 2^{M_n - M_d} / L_d   (Algorithm 1's output
+// ratio with the sets V^l of one instance above and the sets K^l of another below)
+__global__ void two_instance_ratio_kernel(const float* __restrict__ acc_n, const float* __restrict__ ml_n,
+                                          const float* __restrict__ ml_d, __nv_bfloat16* __restrict__ out, int n_heads,
+                                          int d) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_heads * d) return;
+  const int h = i / d;
+  const float Mn = ml_n[2 * h], Md = ml_d[2 * h], Ld = ml_d[2 * h + 1];
+  const float f = (Ld > 0.f && Mn != -INFINITY) ? exp2f(Mn - Md) / Ld : 0.f;
+  out[i] = __float2bfloat16(acc_n[i] * f);
+}
+
+cudaError_t launch_two_instance_ratio(const float* acc_n, const float* ml_n, const float* ml_d, void* out, int n_heads, int d,
+                                      cudaStream_t st) {
+  const int n = n_heads * d;
+  two_instance_ratio_kernel<<<(n + 255) / 256, 256, 0, st>>>(acc_n, ml_n, ml_d, static_cast<__nv_bfloat16*>(out), n_heads, d);
+  return cudaGetLastError();
+}
+
 // Decode attention fused with the append of one token per stream of the layer (k_new, v_new:
 // [B*H, d] bf16; all streams of the layer have the same level-0 fill).  k_new == nullptr: plain decode.
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
@@ -477,7 +524,7 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
   const StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                      new_len};
+                      new_len, nullptr, nullptr};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q),
                                                         static_cast<__nv_bfloat16*>(out), part, tickets, status, ap,
                                                         tm->k, tm->v);

@@ -1,6 +1,6 @@
 """Kernel-level timing of the BalanceKV library on synthetic device data.
 
-    python -m paper_2502_07861_b200.microbench decode   --batch 32 --cache-len 8192 --levels 2
+    python -m paper_2502_07861_b200.microbench decode   --batch 32 --cache-len 8192 --levels 2 [--two-instance]
     python -m paper_2502_07861_b200.microbench compress --streams 8 --context 32768 --block 1024 --levels 2
 
 Prints one JSON line per run.  Inputs are drawn on the device (torch.randn), which is enough
@@ -34,6 +34,9 @@ def run_decode(a):
     bytes_layer = B * H * Lc * 2 * d * esz
     # enough distinct layers that a layer is evicted from L2 (126 MB) before it is read again
     n_layers = max(2, min(a.max_layers, (512 << 20) // max(bytes_layer, 1) + 1))
+    if a.two_instance:          # Algorithm 1 with a separate denominator instance: two slots (caches) per layer
+        n_layers += n_layers % 2
+        bytes_layer *= 2
     ctx = bk.Context(n_seqs=B, n_layers=n_layers, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64,
                      levels=T, max_tokens=Lc << T)
     K = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
@@ -43,21 +46,25 @@ def run_decode(a):
     q = torch.randn(B, H * g, d, device="cuda").to(torch.bfloat16)
     out = torch.empty_like(q)
     raw = int(torch.cuda.current_stream().cuda_stream)
+    if a.two_instance:
+        call = lambda i: ctx.decode_attn_two(2 * (i % (n_layers // 2)), 2 * (i % (n_layers // 2)) + 1, q, out, stream=raw)
+    else:
+        call = lambda i: ctx.decode_attn(i % n_layers, q, out, stream=raw)
     for i in range(3 * n_layers):
-        ctx.decode_attn(i % n_layers, q, out, stream=raw)
+        call(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     iters = a.iters
     e0.record()
     for i in range(iters):
-        ctx.decode_attn(i % n_layers, q, out, stream=raw)
+        call(i)
     e1.record()
     torch.cuda.synchronize()
     us = 1e3 * e0.elapsed_time(e1) / iters
     hbm, _, src = _peaks()
     gbs = bytes_layer / (us * 1e-6) / 1e9
     st = ctx.stats()
-    print(json.dumps(dict(kernel="decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
+    print(json.dumps(dict(kernel="decode_two_instance" if a.two_instance else "decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
                           layers_cycled=n_layers, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
                           peak_gbs=hbm, frac=gbs / hbm, peak_source=src, device_status=st["device_status"])))
     ctx.close()
@@ -121,6 +128,7 @@ def main():
     d.add_argument("--levels", type=int, default=2)
     d.add_argument("--iters", type=int, default=50)
     d.add_argument("--max-layers", type=int, default=16)
+    d.add_argument("--two-instance", action="store_true")
     c = sub.add_parser("compress")
     c.add_argument("--streams", type=int, default=8)
     c.add_argument("--head-dim", type=int, default=128)
