@@ -68,3 +68,18 @@ def test_two_instance_T0_is_exact_attention_and_empty_slots_give_zeros(cuda_lib)
     with pytest.raises(cuda_lib.BalanceKVError):
         cuda_lib.Context(n_seqs=1, n_layers=2, n_kv_heads=1, n_q_heads=1, head_dim=64, dtype="fp32", block=64, levels=0,
                          max_tokens=64).decode_attn_two(0, 1, torch.zeros(1, 1, 64, device="cuda"))
+
+
+def test_error_sweep_point_small_c_beats_uniform_on_clustered_keys(cuda_lib):
+    """One point of the error-against-rate sweep: on near-duplicate keys a small walk constant gives a
+    clearly lower attention error than uniform sampling at the same rate, the paper's constant about
+    the same (its walk is almost a fair coin at these norms)."""
+    from paper_2502_07861_b200 import error_sweep
+
+    acc = {}
+    for seed in range(4):
+        for k, v in error_sweep.run_point("clustered", seed, 2, 4096, 128, 128, 2, 0.25, 0).items():
+            acc[k] = acc.get(k, 0.0) + v / 4
+    assert acc["balancekv_small_c"] < 0.7 * acc["uniform"]
+    assert 0.5 * acc["uniform"] < acc["balancekv_paper_c"] < 2.0 * acc["uniform"]
+    assert acc["balancekv_paper_c_fails"] == 0
