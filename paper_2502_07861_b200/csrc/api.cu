@@ -21,7 +21,8 @@ bool decode_mma_supported(const Geom& G);
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out);
 void decode_mma_release(void* maps);
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
-                                    float* scratch, int splits, int* status, const void* maps, cudaStream_t st);
+                                    float* scratch, int splits, int* status, const void* maps, int keys_only,
+                                    cudaStream_t st);
 cudaError_t launch_two_instance_ratio(const float* acc_n, const float* ml_n, const float* ml_d, void* out, int n_heads, int d,
                                       cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
@@ -673,12 +674,12 @@ int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, co
   {
     ProfScope ps(c, 4, st);
     BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_num, q, acc_n, ml_n, c->d_decode_scratch, pick_splits(c, layer_num),
-                                     c->d_status, c->decode_maps, st));
+                                     c->d_status, c->decode_maps, 0, st));
   }
   {
     ProfScope ps(c, 4, st);
     BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_den, q, acc_d, ml_d, c->d_decode_scratch, pick_splits(c, layer_den),
-                                     c->d_status, c->decode_maps, st));
+                                     c->d_status, c->decode_maps, 1, st));   // the unit values are not read
   }
   BKV_CUDA(launch_two_instance_ratio(acc_n, ml_n, ml_d, out, n_heads, d, st));
   c->kernels_launched += 3;

@@ -108,6 +108,7 @@ struct StepAppend {
   // MergeAndReduce instance by the denominator of another; this is one such part.
   float* raw_acc;
   float* raw_ml;
+  int keys_only;                // 1: only (M, sum) are wanted (a denominator instance): V is neither loaded nor multiplied
 };
 
 struct TileRef {
@@ -172,11 +173,13 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
     unsigned char* st = tiles + (size_t)(i % kStages) * kStageBytes;
     uint64_t* bar = &full[i % kStages];
-    mbar_expect_tx(bar, kStageBytes);
+    mbar_expect_tx(bar, ap.keys_only ? kTensorBytes : kStageBytes);
     tma_load_2d(st, &tmK, 0, (int)tr.row, bar);
     tma_load_2d(st + kHalf, &tmK, 64, (int)tr.row, bar);
-    tma_load_2d(st + kTensorBytes, &tmV, 0, (int)tr.row, bar);
-    tma_load_2d(st + kTensorBytes + kHalf, &tmV, 64, (int)tr.row, bar);
+    if (!ap.keys_only) {
+      tma_load_2d(st + kTensorBytes, &tmV, 0, (int)tr.row, bar);
+      tma_load_2d(st + kTensorBytes + kHalf, &tmV, 64, (int)tr.row, bar);
+    }
   };
   if (tid == 0)
     for (int i = 0; i < min(kStages, my_tiles); ++i) issue(i);
@@ -250,6 +253,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       const uint32_t pl[4] = {pack_bf16(x0 - bf16_lo(ph[0]), x1 - bf16_hi(ph[0])), 0u,
                               pack_bf16(x2 - bf16_lo(ph[2]), x3 - bf16_hi(ph[2])), 0u};
       // ---- O[16 x 128] += P[16 x 16] V[16 x 128]
+      if (!ap.keys_only)
 #pragma unroll
       for (int nb = 0; nb < 8; ++nb) {
         uint32_t vb[4];
@@ -479,14 +483,15 @@ cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const vo
 
 // Un-normalised parts (see StepAppend::raw_acc) of the layer's streams for the two-instance estimator.
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
-                                    float* scratch, int splits, int* status, const void* maps, cudaStream_t st) {
+                                    float* scratch, int splits, int* status, const void* maps, int keys_only,
+                                    cudaStream_t st) {
   if (!maps || !raw_acc || !raw_ml) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml};
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
                                                         tickets, status, ap, tm->k, tm->v);
   return cudaGetLastError();
@@ -524,7 +529,7 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
   const StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                      new_len, nullptr, nullptr};
+                      new_len, nullptr, nullptr, 0};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q),
                                                         static_cast<__nv_bfloat16*>(out), part, tickets, status, ap,
                                                         tm->k, tm->v);

@@ -36,7 +36,7 @@ def run_decode(a):
     n_layers = max(2, min(a.max_layers, (512 << 20) // max(bytes_layer, 1) + 1))
     if a.two_instance:          # Algorithm 1 with a separate denominator instance: two slots (caches) per layer
         n_layers += n_layers % 2
-        bytes_layer *= 2
+        bytes_layer = bytes_layer * 3 // 2      # K and V of the numerator slot, K of the denominator slot
     ctx = bk.Context(n_seqs=B, n_layers=n_layers, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64,
                      levels=T, max_tokens=Lc << T)
     K = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
