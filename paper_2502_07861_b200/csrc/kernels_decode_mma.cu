@@ -150,17 +150,23 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const int splits = gridDim.y, split = blockIdx.y;
   const int64_t stream_base = (int64_t)stream * G.rows_per_stream;
 
-  if (tid <= G.T) {
-    const Seg s = A.seg[(size_t)stream * (G.T + 1) + tid];
-    seg_s[tid] = s;
-    lvl_tiles[tid] = (s.len + kTN - 1) / kTN;
-  }
+  // Launched with programmatic stream serialization, this grid may become resident while the
+  // previous kernel of the stream is still finishing (the launch latency overlaps its tail);
+  // nothing that kernel wrote is touched before the wait below.  Without the launch attribute
+  // both instructions do nothing.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
     for (int s = 0; s <= kStages; ++s) mbar_init(&full[s], 1);       // full[kStages]: the combine's bulk copy
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (tid <= G.T) {
+    const Seg s = A.seg[(size_t)stream * (G.T + 1) + tid];
+    seg_s[tid] = s;
+    lvl_tiles[tid] = (s.len + kTN - 1) / kTN;
   }
   __syncthreads();
   int n_tiles = 0;
@@ -530,10 +536,20 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   dim3 grid(n_sl, splits);
   const StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
                       new_len, nullptr, nullptr, 0};
-  decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q),
-                                                        static_cast<__nv_bfloat16*>(out), part, tickets, status, ap,
-                                                        tm->k, tm->v);
-  return cudaGetLastError();
+  // programmatic stream serialization: back-to-back decode steps overlap a launch with the
+  // previous kernel's tail (see the kernel's prologue)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_mma_kernel, G, A, layer, static_cast<const __nv_bfloat16*>(q),
+                            static_cast<__nv_bfloat16*>(out), part, tickets, status, ap, tm->k, tm->v);
 }
 
 }  // namespace bkv
