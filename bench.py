@@ -107,7 +107,8 @@ class ClockSampler:
 
 def oracle_sample(w, K, V, q, sample_tokens, decode_steps):
     """The oracle, as it stands, on the first `sample_tokens` tokens of every stream plus
-    `decode_steps` decode steps; returns (seconds, token-heads, threads)."""
+    `decode_steps` decode steps; returns (seconds spent, token-heads, threads, seconds with the
+    decode part scaled linearly to all of the workload's decode steps)."""
     import oracle
 
     B, H, d, g = w["n_seqs"], w["n_kv_heads"], w["head_dim"], w["n_q_heads"] // w["n_kv_heads"]
@@ -120,13 +121,15 @@ def oracle_sample(w, K, V, q, sample_tokens, decode_steps):
             o.append(K[b, h, :sample_tokens], V[b, h, :sample_tokens])
             streams.append((b, h, o))
     oracle.compress_streams([s[2] for s in streams])
+    t_ctx = time.perf_counter() - t0
     n_ctx = w["context"]
     for s in range(decode_steps):
         for b, h, o in streams:
             o.append(K[b, h, n_ctx + s:n_ctx + s + 1], V[b, h, n_ctx + s:n_ctx + s + 1])
             o.decode(q[s, b, h * g:(h + 1) * g])
     dt = time.perf_counter() - t0
-    return dt, B * H * sample_tokens, oracle.num_threads()
+    scaled = t_ctx + (dt - t_ctx) * (w["decode_steps"] / decode_steps if decode_steps else 0.0)
+    return dt, B * H * sample_tokens, oracle.num_threads(), scaled
 
 
 def run_reference(args, w):
@@ -140,7 +143,7 @@ def run_reference(args, w):
         oracle_sample(w, K, V, q, w["block"] * 2, 1)
     times = []
     for _ in range(args.steps):
-        dt, units, threads = oracle_sample(w, K, V, q, sample, dsteps)
+        dt, units, threads, _ = oracle_sample(w, K, V, q, sample, dsteps)
         times.append(dt)
     val = units * len(times) / sum(times)
     sample_txt = f"first {sample} of {w['context']} context tokens of each of the {w['n_kv_heads']} streams + {dsteps} decode steps"
@@ -237,12 +240,11 @@ def main():
         flush.fill_(1)
         step_device()
     launches_before = ctx.stats()["kernels_launched"]
-    # per-launch events: every compression-side launch, the context append of each step, and every
-    # 16th decode-attention launch (events around all 256 would slow the loop they measure)
-    dec_stride = 16
-    ctx.profile_enable(True)
-    ctx.profile_sample("decode", dec_stride)
-    ctx.profile_sample("append", n_dec + 1)
+    # per-launch events around every compression-side launch and the context append.  A decode step is
+    # one launch (it attends and appends the step's token), so the events that bracket the decode loop
+    # give that kernel's average launch-to-launch duration; events between the launches would stop
+    # consecutive launches from overlapping their launch latency and slow the loop they measure.
+    ctx.profile_enable(True, classes=("append", "radii", "gram_walk", "compact", "bookkeeping"))
     ctx.profile_read()
     sampler = ClockSampler(local)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -298,15 +300,14 @@ def main():
     cp_bytes = (t // 2) * (2 * 2 * d * esz + 8) + t
     cp_gbs = cp_bytes * n_calls * args.steps / (cp_ms * 1e-3) / 1e9 if cp_n else 0.0
     # decode: every stored row of K and V once per launch
-    dc_n, dc_ms = prof["decode"]
+    dc_n, dc_ms = n_dec * args.steps, float(t_dec.sum())
     stored0 = n_ctx >> T
-    dec_bytes_timed = sum(B * H * (stored0 + s + 1) * 2 * d * esz for s in range(0, n_dec, dec_stride)) * args.steps
+    dec_bytes_timed = sum(B * H * (stored0 + s) * 2 * d * esz for s in range(n_dec)) * args.steps   # rows attended from the cache
     dc_gbs = dec_bytes_timed / (dc_ms * 1e-3) / 1e9 if dc_n else 0.0
 
-    # time share of each kernel class in the timed region (sampled classes scaled to all launches)
+    # time share of each kernel class in the timed region
     dc_launches = n_dec * args.steps
-    # a launch's event bracket also holds the gap to its neighbours, so the loop time bounds the total
-    dc_total_ms = min(dc_ms / max(dc_n, 1) * dc_launches, float(t_dec.sum()))
+    dc_total_ms = dc_ms
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
     # summarised under profiles/ (average of the level-0 and level-1 launches; the decode figure is
     # a cold-L2 launch of the same shape, while this loop re-reads its cache from L2)
@@ -321,7 +322,7 @@ def main():
                     traffic=traffic.get("decode"), ms_per_launch=dc_ms / max(dc_n, 1), launches=dc_launches, launches_timed=dc_n,
                     ms_total=dc_total_ms,
                     note="the cache of this workload (35 MB) stays in L2 between decode steps; HBM-bound shapes are "
-                         "timed by `python -m paper_2502_07861_b200.microbench decode`"))
+                         "timed by `python -m paper_2502_07861_b200.microbench decode`; duration = decode loop time / launches"))
     for k in kernels.values():
         k["share_of_step"] = k["ms_total"] / total_ms
     dominant = max(kernels, key=lambda n: kernels[n]["ms_total"])
@@ -331,10 +332,11 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        sample, dsteps = n_ctx, (max(n_dec // 8, 1) if n_dec else 0)
-        dt, units, threads = oracle_sample(w, Kf, Vf, qf, sample, dsteps)
-        cpu = dict(value=units / dt, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
-                   sample=f"first {sample} of {n_ctx} context tokens of each of the {B * H} streams + {dsteps} decode steps")
+        sample, dsteps = n_ctx, (max(n_dec // 4, 1) if n_dec else 0)
+        dt, units, threads, scaled = oracle_sample(w, Kf, Vf, qf, sample, dsteps)
+        cpu = dict(value=units / scaled, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
+                   sample=f"all {n_ctx} context tokens of each of the {B * H} streams + {dsteps} of the {n_dec} decode steps "
+                          f"(their time scaled to {n_dec})")
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
