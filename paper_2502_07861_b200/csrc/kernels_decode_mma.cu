@@ -332,6 +332,43 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const uint32_t part_bytes = (uint32_t)splits * g * PS * sizeof(float);
   const bool staged = part_bytes <= kStages * kStageBytes - kStageOff;
   const float* sp_s = reinterpret_cast<const float*>(tiles + kStageOff);
+  if (ap.k_new) {
+    // append (every CTA of the stream has taken its ticket, so nobody reads the old segment table
+    // any more): one 256-byte row of K and of V, the position, the new length of C^0.  Done first,
+    // so that the writes drain while the partials are combined.
+    const size_t dst = ((size_t)stream_base + G.region_off[0] + ap.rel_row) * kD;
+    if (tid < 16) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.K) + dst)[tid] =
+        reinterpret_cast<const uint4*>(ap.k_new + (size_t)sl * kD)[tid];
+    else if (tid < 32) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.V) + dst)[tid - 16] =
+        reinterpret_cast<const uint4*>(ap.v_new + (size_t)sl * kD)[tid - 16];
+    else if (tid == 32) {
+      A.idx[stream_base + G.region_off[0] + ap.rel_row] = ap.idx0;
+      A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
+    }
+  }
+  // the appended token's operands are requested now, so that their latency overlaps the staging:
+  // per lane 4 dims of <q_h, k_new> for this warp's (up to two) heads, and this thread's first
+  // four columns of v_new
+  float dot_pre[2] = {0.f, 0.f};
+  uint2 vn_pre = make_uint2(0u, 0u);
+  if (ap.k_new) {
+    const uint2 kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
+    const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&kn.y);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int h = warp + kWarps * hh;
+      if (h < g) {
+        const uint2 qv = *reinterpret_cast<const uint2*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane);
+        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv.y);
+        float d = __bfloat162float(q01.x) * __bfloat162float(k01.x);
+        d = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), d);
+        d = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), d);
+        d = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), d);
+        dot_pre[hh] = d;
+      }
+    }
+    if (tid < g * (kD / 4)) vn_pre = *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + (tid % (kD / 4)) * 4);
+  }
   if (staged) {
     if (tid == 0) {
       // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
@@ -368,12 +405,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     float fN = 0.f;
     if (ap.k_new) {
       // the appended token: level 0, weight 1; <q, k_new> in fp32, 4 dims per lane
-      const __nv_bfloat16* qh = q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane;
-      const __nv_bfloat16* kn = ap.k_new + (size_t)sl * kD + 4 * lane;
-      float dot = 0.f;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) dot = fmaf(__bfloat162float(qh[i]), __bfloat162float(kn[i]), dot);
-      const float x = warp_sum(dot) * sc;
+      const float x = warp_sum(h < kWarps ? dot_pre[0] : dot_pre[1]) * sc;
       const float M2 = fmaxf(M, x);
       const float fS = M == -INFINITY ? 0.f : exp2f(M - M2);
       fN = exp2f(x - M2);
@@ -406,9 +438,10 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     }
     if (ap.k_new) {
       const float fN = cN[h];
-      const __nv_bfloat16* vn = ap.v_new + (size_t)sl * kD + c;
-      acc.x = fmaf(__bfloat162float(vn[0]), fN, acc.x); acc.y = fmaf(__bfloat162float(vn[1]), fN, acc.y);
-      acc.z = fmaf(__bfloat162float(vn[2]), fN, acc.z); acc.w = fmaf(__bfloat162float(vn[3]), fN, acc.w);
+      const uint2 vn = i == tid ? vn_pre : *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + c);
+      const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vn.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vn.y);
+      acc.x = fmaf(__bfloat162float(v01.x), fN, acc.x); acc.y = fmaf(__bfloat162float(v01.y), fN, acc.y);
+      acc.z = fmaf(__bfloat162float(v23.x), fN, acc.z); acc.w = fmaf(__bfloat162float(v23.y), fN, acc.w);
     }
     if (ap.raw_acc) {
       const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
@@ -420,18 +453,6 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c);
     o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
     o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-  }
-  if (ap.k_new) {
-    // append: one 256-byte row of K and of V, the position, the new length of C^0
-    const size_t dst = ((size_t)stream_base + G.region_off[0] + ap.rel_row) * kD;
-    if (tid < 16) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.K) + dst)[tid] =
-        reinterpret_cast<const uint4*>(ap.k_new + (size_t)sl * kD)[tid];
-    else if (tid < 32) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.V) + dst)[tid - 16] =
-        reinterpret_cast<const uint4*>(ap.v_new + (size_t)sl * kD)[tid - 16];
-    else if (tid == 32) {
-      A.idx[stream_base + G.region_off[0] + ap.rel_row] = ap.idx0;
-      A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
-    }
   }
   if (tid == 0) tickets[sl] = 0;   // ready for the next launch
 }
