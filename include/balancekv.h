@@ -205,6 +205,21 @@ int balancekv_stream_append_layer_keys(balancekv_ctx* ctx, int layer, const void
 int balancekv_decode_attn_two(balancekv_ctx* ctx, int layer_num, int layer_den, const void* q, void* out,
                               void* stream);
 
+/* Decode over several layer slots at once:
+ *   out = sum over the slots of layers_num of  sum_i w_i e^{<k_i,q>/sqrt d} v_i
+ *       / sum over the slots of layers_den of  sum_i w_i e^{<k_i,q>/sqrt d}.
+ * With the same slots on both sides this is the estimator of Theorem 3.3 over the union of their
+ * caches -- e.g. the paper's single-layer experiments (Appendix B), which keep the first 256 tokens
+ * exactly: one slot holds them and is never compressed (balancekv_compress_layer leaves the other
+ * slots alone), a second slot runs BalanceKV on the rest with a recent window.  With different
+ * slots it is Algorithm 1's output ratio (numerator instances above, e.g. one per value-norm bucket
+ * that the caller routes tokens to; the denominator instance below).  At most
+ * BALANCEKV_MAX_MERGE distinct slots, none twice on a side; bf16, head_dim 128, group <= 8 only
+ * (else BALANCEKV_E_INVAL).  layers_* are host arrays.  The first call allocates its buffers. */
+#define BALANCEKV_MAX_MERGE 8
+int balancekv_decode_attn_merged(balancekv_ctx* ctx, const int32_t* layers_num, int n_num, const int32_t* layers_den,
+                                 int n_den, const void* q, void* out, void* stream);
+
 /* Kernel timing for roofline reports.  While enabled, every launch of the kernel classes
  * below is bracketed by CUDA events on its launch stream (at most 8192 launches between two
  * reads; later ones are not recorded).  balancekv_profile_read synchronises the device and

@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     OracleStream,
     build,
     compress_streams,
+    merged_estimate,
     num_threads,
     philox4x32_10,
     softmax_balance,

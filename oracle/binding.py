@@ -184,6 +184,19 @@ def two_instance_estimate(numerator_view, denominator_view, q):
     return num * np.exp(mn - md)[:, None] / den[:, None]
 
 
+def merged_estimate(numerator_views, denominator_views, q):
+    """Value sums of several (K, V, w) views over weight sums of several views: the estimator over the
+    union of caches (same views on both sides) or Algorithm 1's ratio (numerator instances above,
+    the denominator instance below)."""
+    q = _f64(q).reshape(-1, numerator_views[0][0].shape[1])
+    nums = [weighted_sums(v[0], v[1], v[2], q) for v in numerator_views if len(v[2])]
+    dens = [weighted_sums(v[0], v[1], v[2], q) for v in denominator_views if len(v[2])]
+    m = np.max(np.stack([x[2] for x in nums + dens]), axis=0)
+    num = sum(x[0] * np.exp(x[2] - m)[:, None] for x in nums)
+    den = sum(x[1] * np.exp(x[2] - m) for x in dens)
+    return num / den[:, None]
+
+
 class OracleStream:
     """One (sequence, layer, KV head) stream driven by MergeAndReduce."""
 

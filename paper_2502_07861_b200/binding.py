@@ -23,7 +23,7 @@ EXPORTS = [
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
-    "balancekv_decode_attn_two",
+    "balancekv_decode_attn_two", "balancekv_decode_attn_merged",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -89,6 +89,7 @@ def load():
     lib.balancekv_profile_sample.argtypes = [vp, ci, ci]
     lib.balancekv_stream_append_layer_keys.argtypes = [vp, ci, vp, ci, vp]
     lib.balancekv_decode_attn_two.argtypes = [vp, ci, ci, vp, vp, vp]
+    lib.balancekv_decode_attn_merged.argtypes = [vp, vp, ci, vp, ci, vp, vp, vp]
     lib.balancekv_profile_read.argtypes = [vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     for name in EXPORTS:
@@ -228,6 +229,18 @@ class Context:
             out = torch.empty_like(q)
         _check(self.lib.balancekv_decode_attn_two(self._h, layer_num, layer_den, self._dev(q, "q"), self._dev(out, "out"),
                                                   _stream_ptr(stream)), "balancekv_decode_attn_two")
+        return out
+
+    def decode_attn_merged(self, layers_num, layers_den, q, out=None, stream=None):
+        """Value sums of the slots layers_num over weight sums of the slots layers_den (see balancekv.h)."""
+        import torch
+
+        if out is None:
+            out = torch.empty_like(q)
+        ln = (C.c_int32 * len(layers_num))(*layers_num)
+        ld = (C.c_int32 * len(layers_den))(*layers_den)
+        _check(self.lib.balancekv_decode_attn_merged(self._h, ln, len(layers_num), ld, len(layers_den), self._dev(q, "q"),
+                                                     self._dev(out, "out"), _stream_ptr(stream)), "balancekv_decode_attn_merged")
         return out
 
     def stream_step_host(self, layer, q_host, k_host, v_host, out_host, stream=None):

@@ -23,8 +23,8 @@ void decode_mma_release(void* maps);
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
                                     float* scratch, int splits, int* status, const void* maps, int keys_only,
                                     cudaStream_t st);
-cudaError_t launch_two_instance_ratio(const float* acc_n, const float* ml_n, const float* ml_d, void* out, int n_heads, int d,
-                                      cudaStream_t st);
+cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, unsigned num_mask, unsigned den_mask,
+                                void* out, int n_heads, int d, cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
                                    int rel_row, int idx0, int new_len, cudaStream_t st);
@@ -104,8 +104,8 @@ struct balancekv_ctx {
   cudaEvent_t step_ev[kStepSlots] = {};
   unsigned long long step_count = 0;
   // two-instance estimator: un-normalised parts of the numerator and denominator instances, unit values
-  float* two_acc = nullptr;             // [B, Hq, d] numerator sums
-  float* two_ml = nullptr;              // [2][B, Hq, 2] (max, sum) of the numerator and of the denominator instance
+  float* two_acc = nullptr;             // [BALANCEKV_MAX_MERGE][B, Hq, d] value sums per merged slot
+  float* two_ml = nullptr;              // [BALANCEKV_MAX_MERGE][B, Hq, 2] (max, sum) per merged slot
   void* unit_V = nullptr;               // rows (1, 0, ..., 0) for balancekv_stream_append_layer_keys
   size_t unit_rows = 0;
 
@@ -655,35 +655,52 @@ int balancekv_stream_append_layer_keys(balancekv_ctx* c, int layer, const void* 
   return append_impl(c, layer_streams(c, layer), 0, K, c->unit_V, nullptr, n_tokens, st, layer);
 }
 
-int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, const void* q, void* out, void* stream) {
-  if (!c || !q || !out || layer_num < 0 || layer_num >= c->cfg.n_layers || layer_den < 0 || layer_den >= c->cfg.n_layers)
-    return BALANCEKV_E_INVAL;
+int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, int n_num, const int32_t* layers_den,
+                                 int n_den, const void* q, void* out, void* stream) {
+  if (!c || !q || !out || !layers_num || !layers_den || n_num < 1 || n_den < 1) return BALANCEKV_E_INVAL;
   if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
   if (!c->decode_maps) return BALANCEKV_E_INVAL;          // bf16, head_dim 128, group <= 8 only
+  // distinct slots in order of first appearance, with the sides they enter
+  int slots[BALANCEKV_MAX_MERGE];
+  unsigned num_mask = 0, den_mask = 0;
+  int n_parts = 0;
+  for (int side = 0; side < 2; ++side) {
+    const int32_t* ls = side ? layers_den : layers_num;
+    for (int i = 0; i < (side ? n_den : n_num); ++i) {
+      if (ls[i] < 0 || ls[i] >= c->cfg.n_layers) return BALANCEKV_E_INVAL;
+      int p = 0;
+      while (p < n_parts && slots[p] != ls[i]) ++p;
+      if (p == n_parts) {
+        if (n_parts == BALANCEKV_MAX_MERGE) return BALANCEKV_E_INVAL;
+        slots[n_parts++] = ls[i];
+      }
+      unsigned& mask = side ? den_mask : num_mask;
+      if ((mask >> p) & 1u) return BALANCEKV_E_INVAL;      // a slot twice on one side
+      mask |= 1u << p;
+    }
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int n_heads = c->cfg.n_seqs * c->cfg.n_q_heads, d = c->cfg.head_dim;
   if (!c->two_acc) {   // first call: buffers for the un-normalised parts (allocates)
-    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_acc), sizeof(float) * (size_t)n_heads * d * 2));
-    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_ml), sizeof(float) * (size_t)n_heads * 4));
-    c->bytes_resident += sizeof(float) * ((size_t)n_heads * d * 2 + (size_t)n_heads * 4);
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_acc), sizeof(float) * (size_t)n_heads * d * BALANCEKV_MAX_MERGE));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_ml), sizeof(float) * (size_t)n_heads * 2 * BALANCEKV_MAX_MERGE));
+    c->bytes_resident += sizeof(float) * (size_t)n_heads * (d + 2) * BALANCEKV_MAX_MERGE;
   }
-  float* acc_n = c->two_acc;
-  float* acc_d = c->two_acc + (size_t)n_heads * d;        // the denominator instance's value sums are not used
-  float* ml_n = c->two_ml;
-  float* ml_d = c->two_ml + (size_t)n_heads * 2;
-  {
+  for (int p = 0; p < n_parts; ++p) {
     ProfScope ps(c, 4, st);
-    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_num, q, acc_n, ml_n, c->d_decode_scratch, pick_splits(c, layer_num),
-                                     c->d_status, c->decode_maps, 0, st));
+    const int keys_only = ((num_mask >> p) & 1u) ? 0 : 1;  // a slot that only enters the denominator: values are not read
+    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, slots[p], q, c->two_acc + (size_t)p * n_heads * d,
+                                     c->two_ml + (size_t)p * n_heads * 2, c->d_decode_scratch, pick_splits(c, slots[p]),
+                                     c->d_status, c->decode_maps, keys_only, st));
   }
-  {
-    ProfScope ps(c, 4, st);
-    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, layer_den, q, acc_d, ml_d, c->d_decode_scratch, pick_splits(c, layer_den),
-                                     c->d_status, c->decode_maps, 1, st));   // the unit values are not read
-  }
-  BKV_CUDA(launch_two_instance_ratio(acc_n, ml_n, ml_d, out, n_heads, d, st));
-  c->kernels_launched += 3;
+  BKV_CUDA(launch_merged_ratio(c->two_acc, c->two_ml, n_parts, num_mask, den_mask, out, n_heads, d, st));
+  c->kernels_launched += n_parts + 1;
   return BALANCEKV_OK;
+}
+
+int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, const void* q, void* out, void* stream) {
+  const int32_t n = layer_num, dn = layer_den;
+  return balancekv_decode_attn_merged(c, &n, 1, &dn, 1, q, out, stream);
 }
 
 int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,

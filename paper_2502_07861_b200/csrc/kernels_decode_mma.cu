@@ -524,23 +524,37 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   return cudaGetLastError();
 }
 
-// out = numerator parts / denominator parts: z = acc_n 2^{M_n - M_d} / L_d   (Algorithm 1's output
-// ratio with the sets V^l of one instance above and the sets K^l of another below)
-__global__ void two_instance_ratio_kernel(const float* __restrict__ acc_n, const float* __restrict__ ml_n,
-                                          const float* __restrict__ ml_d, __nv_bfloat16* __restrict__ out, int n_heads,
-                                          int d) {
+// Ratio of merged parts: the value sums of the numerator slots over the weight sums of the
+// denominator slots,
+//   out = sum_p acc_p 2^{M_p - M*} / sum_r L_r 2^{M_r - M*},   M* the largest M involved
+// (Algorithm 1's output ratio: the union of the numerator instances' sets above, the
+// denominator instance's sets below; with the same slots on both sides, the estimator over the
+// union of their caches).  parts: acc [n_parts][n_heads][d], ml [n_parts][n_heads][2]; num_mask /
+// den_mask: bit p set = part p enters the numerator / the denominator.
+__global__ void merged_ratio_kernel(const float* __restrict__ acc, const float* __restrict__ ml, int n_parts,
+                                    unsigned num_mask, unsigned den_mask, __nv_bfloat16* __restrict__ out, int n_heads,
+                                    int d) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_heads * d) return;
   const int h = i / d;
-  const float Mn = ml_n[2 * h], Md = ml_d[2 * h], Ld = ml_d[2 * h + 1];
-  const float f = (Ld > 0.f && Mn != -INFINITY) ? exp2f(Mn - Md) / Ld : 0.f;
-  out[i] = __float2bfloat16(acc_n[i] * f);
+  float M = -INFINITY;
+  for (int p = 0; p < n_parts; ++p) M = fmaxf(M, ml[((size_t)p * n_heads + h) * 2]);
+  float num = 0.f, den = 0.f;
+  for (int p = 0; p < n_parts; ++p) {
+    const float Mp = ml[((size_t)p * n_heads + h) * 2];
+    if (Mp == -INFINITY) continue;                 // an empty slot
+    const float f = exp2f(Mp - M);
+    if ((num_mask >> p) & 1u) num = fmaf(acc[(size_t)p * n_heads * d + i], f, num);
+    if ((den_mask >> p) & 1u) den = fmaf(ml[((size_t)p * n_heads + h) * 2 + 1], f, den);
+  }
+  out[i] = __float2bfloat16(den > 0.f ? num / den : 0.f);
 }
 
-cudaError_t launch_two_instance_ratio(const float* acc_n, const float* ml_n, const float* ml_d, void* out, int n_heads, int d,
-                                      cudaStream_t st) {
+cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, unsigned num_mask, unsigned den_mask,
+                                void* out, int n_heads, int d, cudaStream_t st) {
   const int n = n_heads * d;
-  two_instance_ratio_kernel<<<(n + 255) / 256, 256, 0, st>>>(acc_n, ml_n, ml_d, static_cast<__nv_bfloat16*>(out), n_heads, d);
+  merged_ratio_kernel<<<(n + 255) / 256, 256, 0, st>>>(acc, ml, n_parts, num_mask, den_mask,
+                                                       static_cast<__nv_bfloat16*>(out), n_heads, d);
   return cudaGetLastError();
 }
 

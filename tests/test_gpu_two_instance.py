@@ -83,3 +83,45 @@ def test_error_sweep_point_small_c_beats_uniform_on_clustered_keys(cuda_lib):
     assert acc["balancekv_small_c"] < 0.7 * acc["uniform"]
     assert 0.5 * acc["uniform"] < acc["balancekv_paper_c"] < 2.0 * acc["uniform"]
     assert acc["balancekv_paper_c_fails"] == 0
+
+
+def test_merged_decode_first_tokens_exact_recent_window_and_compressed_middle(cuda_lib):
+    """The paper's single-layer setting: slot 0 keeps the first 256 tokens and is never compressed,
+    slot 1 runs BalanceKV on the rest with a recent window; decode merges the two slots."""
+    B, H, g, d, t, T, W, sink = 1, 2, 4, 128, 128, 2, 64, 256
+    n = sink + t * 8 + 50
+    K = np.empty((B, H, n, d), np.float32)
+    V = np.empty_like(K)
+    for h in range(H):
+        k, v = synth.stream_kv("llama", 93, 0, 0, h, n, d, "bf16")
+        K[0, h], V[0, h] = synth.round_to(0.06 * k, "bf16"), v
+    hz = Harness(cuda_lib, B=B, L=2, H=H, g=g, d=d, dtype="bf16", t=t, T=T, N=n, W=W, seed=6, c_override=0.75)
+    hz.append_layer(0, K[:, :, :sink], V[:, :, :sink])
+    hz.append_layer(1, K[:, :, sink:], V[:, :, sink:])
+    hz.ctx.compress_layer(1)                                    # slot 0 stays as it is
+    # the oracle side: only slot 1's stream compresses
+    hz.events.append(("compress",))
+    hz.oracle_replay_orig = hz.oracle_replay
+
+    def replay(seq, layer, head, rec=None):
+        saved = hz.events
+        hz.events = [e for e in saved if not (e[0] == "compress" and layer == 0)]
+        try:
+            return hz.oracle_replay_orig(seq, layer, head, rec)
+        finally:
+            hz.events = saved
+
+    hz.oracle_replay = replay
+    hz.check_all(2e-4)
+    assert list(hz.ctx.level_sizes(0, 0, 0)) == [sink, 0, 0]
+    for step in range(2):
+        q = synth.queries(93, 0, step, B, H * g, d, "bf16")
+        out = hz.ctx.decode_attn_merged([0, 1], [0, 1], to_device(q, "bf16")).float().cpu().numpy()
+        for h in range(H):
+            views = [hz.oracles[(0, 0, h)].view(), hz.oracles[(0, 1, h)].view()]
+            assert views[0][2].sum() + views[1][2].sum() == n
+            ref = oracle.merged_estimate(views, views, q[0, h * g:(h + 1) * g])
+            assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3
+    with pytest.raises(cuda_lib.BalanceKVError):
+        hz.ctx.decode_attn_merged([0, 0], [1], to_device(q, "bf16"))
+    assert hz.ctx.stats()["device_status"] == 0

@@ -98,3 +98,42 @@ def test_denominator_discrepancy_inside_the_theorem_3_2_style_bound():
         q *= rng.random() * math.sqrt(r["rk2"]) / np.linalg.norm(q)
         lhs = abs(np.dot(r["eta"], np.exp(K @ q / math.sqrt(d))))
         assert lhs <= math.sqrt(d) * 0.5 * math.exp((q @ q) / (2 * math.sqrt(d)) + r["rk2"] / (2 * math.sqrt(d)))
+
+
+def test_merged_estimate_over_a_partition_equals_the_estimate_over_the_whole_set():
+    """Splitting a weighted set into slots and merging their un-normalised parts changes nothing
+    (up to rounding), whatever the split and however different the slots' largest logits."""
+    rng = np.random.default_rng(5)
+    n, d = 90, 8
+    K, V, w = 3.0 * rng.standard_normal((n, d)), rng.standard_normal((n, d)), 2.0 ** rng.integers(0, 3, n)
+    q = rng.standard_normal((5, d))
+    whole = oracle.weighted_attention(K, V, w, q)
+    cuts = [0, 7, 40, 40, 90]                                  # one slot is empty
+    views = [(K[a:b], V[a:b], w[a:b]) for a, b in zip(cuts[:-1], cuts[1:])]
+    assert np.allclose(oracle.merged_estimate(views, views, q), whole, rtol=1e-12, atol=1e-14)
+    # one numerator and one denominator view: the two-instance form
+    assert np.allclose(oracle.merged_estimate([views[1]], [views[3]], q),
+                       oracle.two_instance_estimate(views[1], views[3], q), rtol=1e-12, atol=1e-14)
+
+
+def test_first_tokens_kept_exactly_beside_a_compressed_middle():
+    """The single-layer setting of Appendix B: the first tokens and a recent window at weight 1, the
+    walk on the tokens in between; every token is counted once, and with T = 0 the result is exact."""
+    rng = np.random.default_rng(6)
+    n, d, t, sink, W = 200, 8, 16, 24, 10
+    K, V = rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    q = rng.standard_normal((3, d))
+    for T in (0, 2):
+        head = OracleStream(OracleParams(d=d, t=t, T=T, layer=0))        # never compressed
+        rest = OracleStream(OracleParams(d=d, t=t, T=T, W=W, layer=1, c_override=0.5))
+        head.append(K[:sink], V[:sink])
+        rest.append(K[sink:], V[sink:])
+        rest.compress()
+        views = [head.view(), rest.view()]
+        assert views[0][2].sum() + views[1][2].sum() == n
+        assert np.all(views[1][2][-W:] == 1.0)
+        z = oracle.merged_estimate(views, views, q)
+        if T == 0:
+            assert np.allclose(z, oracle.weighted_attention(K, V, None, q), rtol=1e-12, atol=1e-14)
+        else:
+            assert len(views[1][3]) < n - sink and np.all(np.isfinite(z))
