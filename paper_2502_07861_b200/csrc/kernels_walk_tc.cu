@@ -235,7 +235,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
   // four MMAs that read it are done, which lengthens the prefetch distance of the column ring.
   uint64_t* full = bars + 0;         // [x][3][h] box h of product x's operand landed in slot s: index 6 x + 2 s + h
   uint64_t* empty = bars + 12;       // [x][3][h] product x no longer reads that box -> producer
-  uint64_t* xdone = bars + 24;       // [x][2] product x of the tile in TMEM buffer b finished -> epilogue
+  uint64_t* xdone = bars + 24;       // [2] both products of the tile in TMEM buffer b finished (one arrival per product) -> epilogue
   uint64_t* tmem_empty = bars + 28;  // [2] all epilogue warps have drained buffer b
   uint32_t* tmem_ptr_s = reinterpret_cast<uint32_t*>(bars + 30);
   int* abort_flag = reinterpret_cast<int*>(tmem_ptr_s + 1);
@@ -246,7 +246,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
 
   if (tid == 0) {
     for (int i = 0; i < 12; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); }
-    for (int i = 0; i < 4; ++i) mbar_init(xdone + i, 1);
+    for (int i = 0; i < 2; ++i) mbar_init(xdone + i, 2);
     for (int i = 0; i < 2; ++i) mbar_init(tmem_empty + i, kEpiWarps);       // one arrival per warp (lane 0 after __syncwarp)
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -333,7 +333,7 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
           if (c < r && !(ok = wait_bar(full + 6 * x + 2 * slot + 1, ph, abort_flag))) break;
           umma_tile_hi(d_tmem, arow, b);
           umma_commit(empty + 6 * x + 2 * slot + 1);
-          umma_commit(xdone + 2 * x + buf);
+          umma_commit(xdone + buf);
         }
       }
     }
@@ -416,7 +416,6 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       for (int c = 0; c < r && ok; ++c, ++tile_it) {
         const int buf = tile_it & 1;
         if (!(ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
-        if (!(ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag))) break;
         tc_fence_after();
         const uint32_t tb = tlane + (uint32_t)buf * 256u;
         // pull this group's 32 columns of both accumulators into registers and hand the TMEM
@@ -434,7 +433,6 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       // ---- diagonal tile
       const int buf = tile_it & 1;
       if (ok) ok = wait_bar(xdone + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag);
-      if (ok) ok = wait_bar(xdone + 2 + buf, (uint32_t)((tile_it >> 1) & 1), abort_flag);
       if (bar_red_or(3, kEpiThreads, !ok)) { ok = false; break; }          // uniform: everybody walks or everybody leaves
       ++tile_it;
       float g[32];
