@@ -304,7 +304,7 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   if (cudaMemset(c->d_fail, 0, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   {
     const int n_sl = f.n_seqs * f.n_kv_heads;
-    c->max_splits = std::max(1, std::min(64, (2 * c->sm_count + n_sl - 1) / n_sl));
+    c->max_splits = std::max(1, std::min(64, 2 * c->sm_count / n_sl));   // two resident CTAs per SM; rounding down keeps one wave
     if (f.decode_splits > 0) c->max_splits = std::min(64, f.decode_splits);
     const size_t sb = decode_scratch_bytes(G, c->max_splits);
     if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->d_decode_scratch), sb))) return fail(rc);

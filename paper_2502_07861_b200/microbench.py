@@ -38,7 +38,7 @@ def run_decode(a):
         n_layers += n_layers % 2
         bytes_layer = bytes_layer * 3 // 2      # K and V of the numerator slot, K of the denominator slot
     ctx = bk.Context(n_seqs=B, n_layers=n_layers, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64,
-                     levels=T, max_tokens=Lc << T)
+                     levels=T, max_tokens=Lc << T, decode_splits=a.splits)
     K = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     V = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     for l in range(n_layers):
@@ -65,7 +65,7 @@ def run_decode(a):
     gbs = bytes_layer / (us * 1e-6) / 1e9
     st = ctx.stats()
     print(json.dumps(dict(kernel="decode_two_instance" if a.two_instance else "decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
-                          layers_cycled=n_layers, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
+                          layers_cycled=n_layers, splits=a.splits, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
                           peak_gbs=hbm, frac=gbs / hbm, peak_source=src, device_status=st["device_status"])))
     ctx.close()
 
@@ -129,6 +129,7 @@ def main():
     d.add_argument("--iters", type=int, default=50)
     d.add_argument("--max-layers", type=int, default=16)
     d.add_argument("--two-instance", action="store_true")
+    d.add_argument("--splits", type=int, default=0, help="split-K factor (0 = automatic)")
     c = sub.add_parser("compress")
     c.add_argument("--streams", type=int, default=8)
     c.add_argument("--head-dim", type=int, default=128)
