@@ -124,7 +124,8 @@ int balancekv_stream_step(balancekv_ctx* ctx, int layer, const void* q, const vo
 /* Same with HOST buffers for q, k_new, v_new and out.  The inputs are read by the CPU during
  * the call (packed into a pinned staging slot of the context and sent as one transfer), so the
  * caller may reuse them as soon as the call returns; out_host is written in stream order
- * (synchronise the stream before reading it).  The first call allocates the staging buffers. */
+ * (synchronise the stream before reading it): a pinned out_host is written by the kernel itself,
+ * pageable memory through a device buffer and a copy.  The first call allocates the staging buffers. */
 int balancekv_stream_step_host(balancekv_ctx* ctx, int layer, const void* q_host, const void* k_host,
                                const void* v_host, void* out_host, void* stream);
 

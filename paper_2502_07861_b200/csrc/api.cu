@@ -765,10 +765,21 @@ int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, 
   std::memcpy(h + qb + kb, v_host, kb);
   BKV_CUDA(cudaMemcpyAsync(c->step_dev_in, h, qb + 2 * kb, cudaMemcpyHostToDevice, st));
   BKV_CUDA(cudaEventRecord(c->step_ev[slot], st));
-  int rc = balancekv_stream_step(c, layer, c->step_dev_in, c->step_dev_in + qb, c->step_dev_in + qb + kb, c->step_dev_out,
-                                 stream);
+  // A pinned (mapped) result buffer is written by the kernel itself: the 8 KB of a step then need
+  // no transfer of their own.  Pageable memory goes through the device buffer and a copy.
+  void* out_dev = nullptr;
+  {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, out_host) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer &&
+        aligned16(at.devicePointer))
+      out_dev = at.devicePointer;
+    else
+      (void)cudaGetLastError();
+  }
+  int rc = balancekv_stream_step(c, layer, c->step_dev_in, c->step_dev_in + qb, c->step_dev_in + qb + kb,
+                                 out_dev ? out_dev : c->step_dev_out, stream);
   if (rc) return rc;
-  BKV_CUDA(cudaMemcpyAsync(out_host, c->step_dev_out, qb, cudaMemcpyDeviceToHost, st));
+  if (!out_dev) BKV_CUDA(cudaMemcpyAsync(out_host, c->step_dev_out, qb, cudaMemcpyDeviceToHost, st));
   return BALANCEKV_OK;
 }
 

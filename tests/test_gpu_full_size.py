@@ -133,7 +133,7 @@ def test_profiler_class_mask_and_sampling(cuda_lib):
 
 
 def test_host_buffer_entry_points_match_the_device_ones(cuda_lib):
-    """append / decode / step through pinned host buffers (more steps than staging slots) give
+    """append / decode / step through host buffers (pinned, one step pageable; more steps than staging slots) give
     bit-identical caches and outputs to the device-pointer calls."""
     Bs, Hs, g, d, n, steps = 2, 2, 4, 128, 200, 70
     mk = lambda: cuda_lib.Context(n_seqs=Bs, n_layers=1, n_kv_heads=Hs, n_q_heads=Hs * g, head_dim=d, dtype="bf16",
@@ -154,8 +154,12 @@ def test_host_buffer_entry_points_match_the_device_ones(cuda_lib):
     qs, ks, vs = bf((steps, Bs, Hs * g, d)).pin_memory(), bf((steps, Bs, Hs, 1, d)).pin_memory(), bf((steps, Bs, Hs, 1, d)).pin_memory()
     outs_h = torch.empty_like(qs).pin_memory()
     out_d = torch.empty(Bs, Hs * g, d, dtype=torch.bfloat16, device="cuda")
+    pageable = torch.empty_like(qs[0])                      # not pinned: goes through the device buffer and a copy
     for s in range(steps):
-        b.stream_step_host(0, qs[s], ks[s], vs[s], outs_h[s])
+        b.stream_step_host(0, qs[s], ks[s], vs[s], pageable if s == 1 else outs_h[s])
+        if s == 1:
+            torch.cuda.synchronize()
+            outs_h[1].copy_(pageable)
     for s in range(steps):
         a.stream_step(0, qs[s].cuda(), ks[s].cuda(), vs[s].cuda(), out_d)
         if s in (0, steps // 2, steps - 1):
