@@ -233,3 +233,32 @@ def test_loaded_cache_decode_sweep_shape(cuda_lib):
                 ref = oracle.weighted_attention(K[b, 0, h], V[b, 0, h], np.full(Lc, 2.0 ** T), q[b, h * g:(h + 1) * g])
                 assert rel_l2(out[b, h * g:(h + 1) * g], ref) <= DEC_TOL["bf16"]
         ctx.close()
+
+
+@pytest.mark.parametrize("gram", [1, 2])
+def test_degenerate_inputs_zero_values_and_duplicate_tokens(cuda_lib, gram):
+    """All-zero values (r_value = 0: the kernel vanishes and the signs are the coins alone) and
+    identical tokens (Ghat = 1 everywhere: with a small constant every other step hits the FAIL clamp,
+    and both sides must count the same FAILs)."""
+    B, L, H, g, d, t = 1, 2, 1, 2, 128, 128
+    n = t * 4
+    K, V = _layer_inputs("llama", 61, B, L, H, n, d, "bf16", key_scale=0.06)
+    V[:, 0] = 0.0                                              # layer 0: zero values
+    K[:, 1] = K[:, 1, :, :1]                                   # layer 1: every token equals the first one
+    V[:, 1] = V[:, 1, :, :1]
+    hz = Harness(cuda_lib, B=B, L=L, H=H, g=g, d=d, dtype="bf16", t=t, T=2, N=n, seed=8, c_override=0.3, gram_path=gram)
+    for l in range(L):
+        hz.append_layer(l, K[:, l], V[:, l])
+    hz.compress()
+    hz.check_all(S_TOL["bf16"])
+    zero = hz.oracles[(0, 0, 0)].calls()
+    assert all(np.all(c["S"] == 0) and np.all(c["p"] == 0.5) for c in zero)
+    dup_fails = sum(c["fails"] for c in hz.oracles[(0, 1, 0)].calls())
+    assert dup_fails >= 0.4 * sum(len(c["eta"]) for c in hz.oracles[(0, 1, 0)].calls())   # every other step: S swings past c and back
+    assert hz.ctx.stats()["walk_fails"] == dup_fails + sum(c["fails"] for c in zero)
+    for l in range(L):
+        q = synth.queries(61, l, 0, B, H * g, d, "bf16")
+        if l == 0:
+            assert np.all(hz.ctx.decode_attn(0, to_device(q, "bf16")).float().cpu().numpy() == 0)
+        else:
+            hz.check_decode(l, q, DEC_TOL["bf16"])
