@@ -117,11 +117,17 @@ radii_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, CallStat* __re
     for (int e = lane; e < G.d; e += 32) mu2 += mu[e] * mu[e];
     mu2 = warp_sum(mu2);
   }
-  for (int r = blockIdx.y * 64 + warp; r < min(G.t, (int)(blockIdx.y + 1) * 64); r += 8) {
-    const char* krow = static_cast<const char*>(A.K) + (size_t)(C.src_row + r) * G.d * esz;
-    const char* vrow = static_cast<const char*>(A.V) + (size_t)(C.src_row + r) * G.d * esz;
+  // d / 8 lanes share a row (8 elements each): with d = 128 a warp works on two rows at a time
+  const int lpr = G.d / 8 < 32 ? G.d / 8 : 32;     // lanes per row
+  const int rpw = 32 / lpr;                        // rows per warp step
+  const int sub = lane / lpr, l0 = lane % lpr;
+  const int row_end = min(G.t, (int)(blockIdx.y + 1) * 64);
+  for (int r = blockIdx.y * 64 + warp * rpw + sub; r - sub < row_end; r += 8 * rpw) {
+    const bool live = r < row_end;
+    const char* krow = static_cast<const char*>(A.K) + (size_t)(C.src_row + (live ? r : 0)) * G.d * esz;
+    const char* vrow = static_cast<const char*>(A.V) + (size_t)(C.src_row + (live ? r : 0)) * G.d * esz;
     float sk = 0.f, sv = 0.f, sm = 0.f;
-    for (int e = lane * 8; e < G.d; e += 256) {
+    for (int e = l0 * 8; e < G.d; e += lpr * 8) {
       float a[8], b[8];
       load8<kBf16>(krow, e, a);
       load8<kBf16>(vrow, e, b);
@@ -132,15 +138,19 @@ radii_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, CallStat* __re
         if (mu) sm = fmaf(a[i], mu[e + i], sm);
       }
     }
-    sk = warp_sum(sk); sv = warp_sum(sv);
+    for (int o = lpr / 2; o > 0; o >>= 1) {
+      sk += __shfl_xor_sync(0xffffffffu, sk, o);
+      sv += __shfl_xor_sync(0xffffffffu, sv, o);
+      if (mu) sm += __shfl_xor_sync(0xffffffffu, sm, o);
+    }
     if (mu) {
-      sm = warp_sum(sm);
       const float shift = sm - 0.5f * mu2;
       sk = fmaxf(sk - 2.f * shift, 0.f);
-      if (lane == 0) tok_shift[(size_t)blockIdx.x * G.t + r] = shift;
+      if (live && l0 == 0) tok_shift[(size_t)blockIdx.x * G.t + r] = shift;
     }
-    mk = fmaxf(mk, sk); mv = fmaxf(mv, sv);
+    if (live) { mk = fmaxf(mk, sk); mv = fmaxf(mv, sv); }
   }
+  mk = warp_max(mk); mv = warp_max(mv);
   __shared__ float smk[8], smv[8];
   if (lane == 0) { smk[warp] = mk; smv[warp] = mv; }
   __syncthreads();
