@@ -288,6 +288,8 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->A.K), (size_t)c->total_rows * row_bytes))) return fail(rc);
   if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->A.V), (size_t)c->total_rows * row_bytes))) return fail(rc);
   if ((rc = dev_alloc(c, &c->A.idx, (size_t)c->total_rows))) return fail(rc);
+  if ((rc = dev_alloc(c, &c->A.nrm, (size_t)c->total_rows))) return fail(rc);
+  if (cudaMemset(c->A.nrm, 0, sizeof(float2) * (size_t)c->total_rows) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   if ((rc = dev_alloc(c, &c->A.seg, (size_t)c->n_streams * (T + 1)))) return fail(rc);
   if (cudaMemset(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (T + 1)) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   // rows that were never written must hold finite numbers: tiles of the decode kernels may
@@ -341,7 +343,7 @@ int balancekv_destroy(balancekv_ctx* c) {
   cudaDeviceSynchronize();
   walk_tc_release(c->tmaps);
   decode_mma_release(c->decode_maps);
-  void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
+  void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->A.nrm, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
                   c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
                   c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->unit_V};
   for (void* p : ptrs)
@@ -497,7 +499,9 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
       int rc = ring_push(c, calls.data() + first, (size_t)n * sizeof(CallDesc), st, &d_calls);
       if (rc) return rc;
       const CallDesc* dc = static_cast<const CallDesc*>(d_calls);
-      const bool need_radii = G.center_keys || G.fixed_rk2 <= 0.f || G.fixed_rv2 <= 0.f;
+      // the tensor-core walk kernel takes the radii from the stored row norms itself
+      const bool need_radii = (G.center_keys || G.fixed_rk2 <= 0.f || G.fixed_rv2 <= 0.f) &&
+                              !(c->use_tc && !G.center_keys && c->A.nrm);
       if (need_radii) {
         ProfScope ps(c, 1, st);
         BKV_CUDA(launch_radii(G, c->A, dc, n, c->d_stats, c->d_tokshift, st));

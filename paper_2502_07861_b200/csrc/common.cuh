@@ -130,6 +130,7 @@ struct Arena {
   void* V;
   int32_t* idx;     // [n_streams * R] original token position
   Seg* seg;         // [n_streams, T+1]
+  float2* nrm;      // [n_streams * R] (||k||^2, ||v||^2) of every stored row, written with the row (null: not kept)
 };
 
 cudaError_t launch_append(const Geom& G, const Arena& A, const AppendDesc* descs, int n_desc, int max_rows,

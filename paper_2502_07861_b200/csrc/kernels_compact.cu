@@ -88,7 +88,10 @@ compact_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, const int8_t
     char* dst = static_cast<char*>(which ? A.V : A.K) + (size_t)(C.dst_row + o) * G.d * esz;
     reinterpret_cast<uint4*>(dst)[ch] = reinterpret_cast<const uint4*>(src)[ch];
   }
-  for (int i = threadIdx.x; i < rows; i += kThreads) A.idx[C.dst_row + o0 + i] = A.idx[C.src_row + kept_pos[o0 + i]];
+  for (int i = threadIdx.x; i < rows; i += kThreads) {
+    A.idx[C.dst_row + o0 + i] = A.idx[C.src_row + kept_pos[o0 + i]];
+    if (A.nrm) A.nrm[C.dst_row + o0 + i] = A.nrm[C.src_row + kept_pos[o0 + i]];
+  }
 }
 
 }  // namespace

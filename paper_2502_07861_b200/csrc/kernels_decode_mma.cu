@@ -336,13 +336,26 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     // append (every CTA of the stream has taken its ticket, so nobody reads the old segment table
     // any more): one 256-byte row of K and of V, the position, the new length of C^0.  Done first,
     // so that the writes drain while the partials are combined.
-    const size_t dst = ((size_t)stream_base + G.region_off[0] + ap.rel_row) * kD;
-    if (tid < 16) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.K) + dst)[tid] =
-        reinterpret_cast<const uint4*>(ap.k_new + (size_t)sl * kD)[tid];
-    else if (tid < 32) reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(A.V) + dst)[tid - 16] =
-        reinterpret_cast<const uint4*>(ap.v_new + (size_t)sl * kD)[tid - 16];
-    else if (tid == 32) {
-      A.idx[stream_base + G.region_off[0] + ap.rel_row] = ap.idx0;
+    const size_t dst_row = (size_t)stream_base + G.region_off[0] + ap.rel_row;
+    if (warp == 0) {                                          // lanes 0-15: the row of K, lanes 16-31: the row of V
+      const __nv_bfloat16* src = (lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD;
+      __nv_bfloat16* dstp = static_cast<__nv_bfloat16*>(lane < 16 ? A.K : A.V) + dst_row * kD;
+      const uint4 v = reinterpret_cast<const uint4*>(src)[lane & 15];
+      reinterpret_cast<uint4*>(dstp)[lane & 15] = v;
+      float s2 = 0.f;                                         // ||k||^2 / ||v||^2 travel with the row
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h2[i]);
+        s2 = fmaf(f.x, f.x, s2);
+        s2 = fmaf(f.y, f.y, s2);
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+      const float v2 = __shfl_sync(0xffffffffu, s2, 16);
+      if (lane == 0 && A.nrm) A.nrm[dst_row] = make_float2(s2, v2);
+    } else if (tid == 32) {
+      A.idx[dst_row] = ap.idx0;
       A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
     }
   }

@@ -16,6 +16,67 @@ __device__ inline void copy_rows(uint4* __restrict__ dst, const uint4* __restric
   for (int i = threadIdx.x; i < total; i += blockDim.x) dst[i] = src[i];
 }
 
+template <bool kBf16>
+__device__ inline float sumsq16(const uint4& v) {
+  float s = 0.f;
+  if (kBf16) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(h[i]);
+      s = fmaf(f.x, f.x, s);
+      s = fmaf(f.y, f.y, s);
+    }
+  } else {
+    const float* f = reinterpret_cast<const float*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s = fmaf(f[i], f[i], s);
+  }
+  return s;
+}
+
+// Copies rows of K and V and records (||k||^2, ||v||^2) of every row: the radii of Algorithm 2
+// (r_key, r_value of a call) then need the norms only, not the rows.  `chunks` (16-byte pieces
+// of a row: 8, 16 or 32) consecutive lanes share a row; blockDim is a multiple of 32.
+template <bool kBf16>
+__device__ inline void copy_rows_norm(uint4* __restrict__ dK, const uint4* __restrict__ sK, uint4* __restrict__ dV,
+                                      const uint4* __restrict__ sV, float2* __restrict__ nrm, int rows, int chunks) {
+  const int total = rows * chunks;
+  for (int i0 = 0; i0 < total; i0 += blockDim.x) {      // whole warps take part in the shuffles
+    const int i = i0 + threadIdx.x;
+    float k2 = 0.f, v2 = 0.f;
+    if (i < total) {
+      const uint4 a = sK[i], b = sV[i];
+      dK[i] = a;
+      dV[i] = b;
+      k2 = sumsq16<kBf16>(a);
+      v2 = sumsq16<kBf16>(b);
+    }
+    for (int o = chunks / 2; o > 0; o >>= 1) {
+      k2 += __shfl_xor_sync(0xffffffffu, k2, o);
+      v2 += __shfl_xor_sync(0xffffffffu, v2, o);
+    }
+    if (i < total && i % chunks == 0) nrm[i / chunks] = make_float2(k2, v2);
+  }
+}
+
+__device__ inline void copy_rows_kv(const Geom& G, const Arena& A, size_t dst_b, int64_t dst_row, const void* Ksrc,
+                                    const void* Vsrc, size_t src_b, int rows) {
+  const int esz = G.is_bf16 ? 2 : 4;
+  const int chunks = G.d * esz / 16;
+  uint4* dK = reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b);
+  uint4* dV = reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b);
+  const uint4* sK = reinterpret_cast<const uint4*>(static_cast<const char*>(Ksrc) + src_b);
+  const uint4* sV = reinterpret_cast<const uint4*>(static_cast<const char*>(Vsrc) + src_b);
+  if (A.nrm && chunks <= 32) {
+    if (G.is_bf16) copy_rows_norm<true>(dK, sK, dV, sV, A.nrm + dst_row, rows, chunks);
+    else copy_rows_norm<false>(dK, sK, dV, sV, A.nrm + dst_row, rows, chunks);
+  } else {
+    copy_rows(dK, sK, rows, chunks);
+    copy_rows(dV, sV, rows, chunks);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 append_kernel(Geom G, Arena A, const AppendDesc* __restrict__ descs, const void* __restrict__ Ksrc,
               const void* __restrict__ Vsrc, const int32_t* __restrict__ idx_src) {
@@ -24,13 +85,9 @@ append_kernel(Geom G, Arena A, const AppendDesc* __restrict__ descs, const void*
   if (row0 < D.n) {
     const int rows = min(kCopyRows, D.n - row0);
     const int esz = G.is_bf16 ? 2 : 4;
-    const int chunks = G.d * esz / 16;
     const size_t dst_b = (size_t)(D.dst_row + row0) * G.d * esz;
     const size_t src_b = ((size_t)D.src_off + (size_t)row0 * G.d) * esz;
-    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b),
-              reinterpret_cast<const uint4*>(static_cast<const char*>(Ksrc) + src_b), rows, chunks);
-    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
-              reinterpret_cast<const uint4*>(static_cast<const char*>(Vsrc) + src_b), rows, chunks);
+    copy_rows_kv(G, A, dst_b, D.dst_row + row0, Ksrc, Vsrc, src_b, rows);
     for (int i = threadIdx.x; i < rows; i += blockDim.x)
       A.idx[D.dst_row + row0 + i] = idx_src ? idx_src[D.src_off / G.d + row0 + i] : D.idx0 + row0 + i;
   }
@@ -49,13 +106,9 @@ append_uniform_kernel(Geom G, Arena A, int layer, int level, int rel_row, int id
   if (row0 < n) {
     const int rows = min(kCopyRows, n - row0);
     const int esz = G.is_bf16 ? 2 : 4;
-    const int chunks = G.d * esz / 16;
     const size_t dst_b = (size_t)(dst_row + row0) * G.d * esz;
     const size_t src_b = ((size_t)sl * n + row0) * G.d * esz;
-    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.K) + dst_b),
-              reinterpret_cast<const uint4*>(static_cast<const char*>(Ksrc) + src_b), rows, chunks);
-    copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
-              reinterpret_cast<const uint4*>(static_cast<const char*>(Vsrc) + src_b), rows, chunks);
+    copy_rows_kv(G, A, dst_b, dst_row + row0, Ksrc, Vsrc, src_b, rows);
     for (int i = threadIdx.x; i < rows; i += blockDim.x)
       A.idx[dst_row + row0 + i] = idx_src ? idx_src[(size_t)sl * n + row0 + i] : idx0 + row0 + i;
   }
@@ -76,7 +129,10 @@ move_kernel(Geom G, Arena A, const MoveDesc* __restrict__ descs) {
               reinterpret_cast<const uint4*>(static_cast<const char*>(A.K) + src_b), rows, chunks);
     copy_rows(reinterpret_cast<uint4*>(static_cast<char*>(A.V) + dst_b),
               reinterpret_cast<const uint4*>(static_cast<const char*>(A.V) + src_b), rows, chunks);
-    for (int i = threadIdx.x; i < rows; i += blockDim.x) A.idx[D.dst_row + row0 + i] = A.idx[D.src_row + row0 + i];
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) {
+      A.idx[D.dst_row + row0 + i] = A.idx[D.src_row + row0 + i];
+      if (A.nrm) A.nrm[D.dst_row + row0 + i] = A.nrm[D.src_row + row0 + i];
+    }
   }
 }
 
@@ -162,6 +218,29 @@ radii_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, CallStat* __re
   }
 }
 
+// r_key^2, r_value^2 of a call from the stored row norms: one CTA per call.
+__global__ void __launch_bounds__(256)
+radii_norms_kernel(Geom G, Arena A, const CallDesc* __restrict__ calls, CallStat* __restrict__ stats) {
+  const CallDesc C = calls[blockIdx.x];
+  float mk = 0.f, mv = 0.f;
+  for (int j = threadIdx.x; j < G.t; j += 256) {
+    const float2 n = A.nrm[C.src_row + j];
+    mk = fmaxf(mk, n.x);
+    mv = fmaxf(mv, n.y);
+  }
+  mk = warp_max(mk); mv = warp_max(mv);
+  __shared__ float smk[8], smv[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { smk[warp] = mk; smv[warp] = mv; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) { mk = fmaxf(mk, smk[w]); mv = fmaxf(mv, smv[w]); }
+    CallStat S{};
+    S.rk2 = mk; S.rv2 = mv;
+    stats[blockIdx.x] = S;
+  }
+}
+
 __global__ void fill_weights_kernel(float* w, int n, float value) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) w[i] = value;
@@ -200,6 +279,10 @@ cudaError_t launch_move(const Geom& G, const Arena& A, const MoveDesc* descs, in
 cudaError_t launch_radii(const Geom& G, const Arena& A, const CallDesc* calls, int n_calls, CallStat* stats,
                          float* tok_shift, cudaStream_t st) {
   if (n_calls <= 0) return cudaSuccess;
+  if (!G.center_keys && A.nrm) {     // the norms were recorded when the rows were written
+    radii_norms_kernel<<<n_calls, 256, 0, st>>>(G, A, calls, stats);
+    return cudaGetLastError();
+  }
   cudaError_t e = cudaMemsetAsync(stats, 0, sizeof(CallStat) * (size_t)n_calls, st);
   if (e != cudaSuccess) return e;
   float* mean = nullptr;

@@ -219,8 +219,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const CallStat* __restrict__ stats,
                const float* __restrict__ tok_shift, int8_t* __restrict__ eta_out, int8_t* __restrict__ dbg_eta,
                float* __restrict__ dbg_S, float* __restrict__ dbg_p, unsigned long long* __restrict__ fail_count,
-               int* __restrict__ status, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV) {
+               int* __restrict__ status, const float2* __restrict__ row_norms,
+               const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int t = G.t, P = t / kTile;
@@ -345,9 +345,6 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
     const int wg = warp >> 2;
     const int q = warp & 3;                   // quarter of the panel = TMEM lane quadrant
     const int row = 32 * q + lane;
-    const float rk2 = G.fixed_rk2 > 0.f ? G.fixed_rk2 : stats[call].rk2;
-    const float rv2 = G.fixed_rv2 > 0.f ? G.fixed_rv2 : stats[call].rv2;
-    const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
     const float scale = 1.4426950408889634f * G.inv_sqrt_d;
     const float cw = G.c;
     const uint32_t tlane = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * wg);
@@ -401,8 +398,33 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       const int head = C.stream % G.H, layer = (C.stream / G.H) % G.L, seq = C.stream / (G.H * G.L);
       for (int i = tid; i < t; i += kEpiThreads)
         thr_s[i] = cw * (1.0f - 2.0f * walk_uniform(G.seed + (uint64_t)seq, layer, head, C.ordinal, level, i));
+      // r_key^2, r_value^2 of the call (inputs of Algorithm 2) = maxima of the stored row norms,
+      // unless a separate kernel has put them (key centering changes them) or they are fixed
+      if (row_norms) {
+        float mk = 0.f, mv = 0.f;
+        for (int i = tid; i < t; i += kEpiThreads) {
+          const float2 n2 = row_norms[C.src_row + i];
+          mk = fmaxf(mk, n2.x);
+          mv = fmaxf(mv, n2.y);
+        }
+        mk = warp_max(mk); mv = warp_max(mv);
+        if (lane == 0) { xs[2 * warp] = mk; xs[2 * warp + 1] = mv; }
+      }
       bar_sync(3, kEpiThreads);
     }
+    float rk2 = G.fixed_rk2, rv2 = G.fixed_rv2;
+    if (row_norms) {
+      float mk = 0.f, mv = 0.f;
+#pragma unroll
+      for (int w = 0; w < kEpiWarps; ++w) { mk = fmaxf(mk, xs[2 * w]); mv = fmaxf(mv, xs[2 * w + 1]); }
+      if (rk2 <= 0.f) rk2 = mk;
+      if (rv2 <= 0.f) rv2 = mv;
+      bar_sync(3, kEpiThreads);                               // xs is reused by the first walk
+    } else {
+      if (rk2 <= 0.f) rk2 = stats[call].rk2;
+      if (rv2 <= 0.f) rv2 = stats[call].rv2;
+    }
+    const float inv_rv2 = rv2 > 0.f ? 1.0f / rv2 : 0.f;
     // All waits of a panel come before its vote barrier (id 3); a thread whose wait timed out
     // skips to the vote, where everybody learns of it and leaves.  The sweep barriers (ids 1, 2)
     // come after the vote and contain no waits, so no thread can be left waiting at them.
@@ -591,17 +613,16 @@ cudaError_t launch_walk_tc(const Geom& G, const Arena& A, const CallDesc* calls,
                            const CallStat* stats, const float* tok_shift, int8_t* eta, int8_t* dbg_eta,
                            float* dbg_S, float* dbg_p, unsigned long long* fail_count, int* status,
                            const void* tmaps, const void*, cudaStream_t st) {
-  (void)A;
   if (n_calls <= 0) return cudaSuccess;
   if (!tmaps) return cudaErrorInvalidValue;
   const TensorMaps* tm = static_cast<const TensorMaps*>(tmaps);
   const size_t smem = tc_smem_bytes(G.t);
   if (G.center_keys)
     walk_tc_kernel<true><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
-                                                          fail_count, status, tm->k, tm->v);
+                                                          fail_count, status, G.center_keys ? nullptr : A.nrm, tm->k, tm->v);
   else
     walk_tc_kernel<false><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
-                                                           fail_count, status, tm->k, tm->v);
+                                                           fail_count, status, G.center_keys ? nullptr : A.nrm, tm->k, tm->v);
   return cudaGetLastError();
 }
 
