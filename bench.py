@@ -297,7 +297,7 @@ def main():
     tensor_ach = flop_per_call * calls_per_launch / (gw_ms_per_launch * 1e-3) / 1e12 if gw_n else 0.0
     # compaction: per call read t/2 rows of K and V, write t/2 rows, t sign bytes, 2 index words per survivor
     cp_n, cp_ms = prof["compact"]
-    cp_bytes = (t // 2) * (2 * 2 * d * esz + 8) + t
+    cp_bytes = (t // 2) * (2 * 2 * d * esz + 8 + 16) + t      # rows, position (4+4 B), norms (8+8 B) per survivor, sign bytes
     cp_gbs = cp_bytes * n_calls * args.steps / (cp_ms * 1e-3) / 1e9 if cp_n else 0.0
     # decode: every stored row of K and V once per launch
     dc_n, dc_ms = n_dec * args.steps, float(t_dec.sum())

@@ -103,7 +103,7 @@ def run_compress(a):
     cp_n, cp_ms = prof["compact"]
     hbm, tf, src = _peaks()
     tfl = flop * a.iters / (gw_ms * 1e-3) / 1e12 if gw_ms else 0.0
-    cp_bytes = n_calls * ((t // 2) * (4 * d * 2 + 8) + t)
+    cp_bytes = n_calls * ((t // 2) * (4 * d * 2 + 8 + 16) + t)   # rows, position, norms per survivor, sign bytes
     cp_gbs = cp_bytes * a.iters / (cp_ms * 1e-3) / 1e9 if cp_ms else 0.0
     st = ctx.stats()
     print(json.dumps(dict(kernel="compress", streams=S, context=n, block=t, levels=T, calls=n_calls,
