@@ -311,7 +311,7 @@ def main():
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
     # summarised under profiles/ (average of the level-0 and level-1 launches; the decode figure is
     # a cold-L2 launch of the same shape, while this loop re-reads its cache from L2)
-    traffic = dict(gram_walk=103.2e6, compact=64.2e6, decode=33.65e6) if (n_ctx, t, T, B * H) == (32768, 1024, 2, 8) else {}
+    traffic = dict(gram_walk=105.4e6, compact=67.5e6, decode=33.65e6) if (n_ctx, t, T, B * H) == (32768, 1024, 2, 8) else {}
     kernels = dict(
         gram_walk=dict(bound="tensor", achieved=tensor_ach, peak=peaks["tensor"], unit="TFLOP/s",
                        frac=tensor_ach / peaks["tensor"], traffic=traffic.get("gram_walk"), ms_per_launch=gw_ms_per_launch, launches=gw_n,
