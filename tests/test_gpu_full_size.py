@@ -167,3 +167,37 @@ def test_host_buffer_entry_points_match_the_device_ones(cuda_lib):
             assert torch.equal(out_d.cpu(), outs_h[s])
     for h in range(Hs):
         assert all(torch.equal(x, y) for x, y in zip(a.cache_view(1, 0, h), b.cache_view(1, 0, h)))
+
+
+def test_tokens_appended_by_decode_steps_compress_like_appended_ones(cuda_lib):
+    """More decode steps than a block, then compress: the rows (and the row norms from which the radii
+    of Algorithm 2 are taken) written by the fused decode step must be those an append writes --
+    same running correlations S_j, bit for bit, and same caches."""
+    Bs, Hs, g, d, t, n0, steps = 1, 2, 4, 128, 64, 100, 160
+    mk = lambda: cuda_lib.Context(n_seqs=Bs, n_layers=1, n_kv_heads=Hs, n_q_heads=Hs * g, head_dim=d, dtype="bf16",
+                                  block=t, levels=2, max_tokens=n0 + steps, seed=2, c_override=0.6)
+    rng = np.random.default_rng(3)
+    K = to_device(0.08 * rng.standard_normal((Bs, Hs, n0 + steps, d)).astype(np.float32), "bf16")
+    V = to_device(rng.standard_normal((Bs, Hs, n0 + steps, d)).astype(np.float32), "bf16")
+    q = to_device(rng.standard_normal((Bs, Hs * g, d)).astype(np.float32), "bf16")
+    a, b = mk(), mk()
+    for c in (a, b):
+        c.debug_enable(True)
+        c.stream_append_layer(0, K[:, :, :n0].contiguous(), V[:, :, :n0].contiguous())
+        c.compress()
+    out = torch.empty_like(q)
+    for s in range(steps):
+        a.stream_step(0, q, K[:, :, n0 + s:n0 + s + 1].contiguous(), V[:, :, n0 + s:n0 + s + 1].contiguous(), out)
+    b.stream_append_layer(0, K[:, :, n0:].contiguous(), V[:, :, n0:].contiguous())
+    a.compress()
+    b.compress()
+    blocks = (n0 + steps) // t
+    for h in range(Hs):
+        assert all(torch.equal(x, y) for x, y in zip(a.cache_view(0, 0, h), b.cache_view(0, 0, h)))
+        for lvl in range(2):
+            for o in range(blocks >> lvl):
+                ea, Sa, _ = a.debug_call(0, 0, h, lvl, o)
+                eb, Sb, _ = b.debug_call(0, 0, h, lvl, o)
+                assert torch.equal(ea, eb) and torch.equal(Sa, Sb)
+    assert torch.equal(a.decode_attn(0, q), b.decode_attn(0, q))
+    assert a.stats()["device_status"] == 0 and a.stats()["calls_run"] == Hs * (blocks + blocks // 2)
