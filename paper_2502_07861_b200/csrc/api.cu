@@ -27,7 +27,7 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
                                 void* out, int n_heads, int d, cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
 cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                               int splits, int* status, const void* maps, cudaStream_t st);
 }  // namespace bkv
@@ -583,6 +583,24 @@ int balancekv_compress_layer(balancekv_ctx* c, int layer, int T, void* stream) {
   return compress_streams(c, layer_streams(c, layer), T, static_cast<cudaStream_t>(stream));
 }
 
+// The layer's segment table as the host mirrors it, if all its streams hold the same segments
+// (lockstep streams): out[l] = (start, len) of level l.  False if they differ.
+static bool layer_seg_hint(balancekv_ctx* c, int layer, Seg* out) {
+  const int T = c->cfg.levels;
+  const std::vector<int>& streams = layer_streams(c, layer);
+  const StreamState& S0 = c->st[streams[0]];
+  for (int s : streams) {
+    const StreamState& S = c->st[s];
+    if (S.start0 != S0.start0 || S.len0 != S0.len0) return false;
+    for (int l = 1; l <= T; ++l)
+      if (S.lvl_len[l] != S0.lvl_len[l] || (l < T && S.lvl_base[l] != S0.lvl_base[l])) return false;
+  }
+  out[0] = Seg{S0.start0, S0.len0};
+  for (int l = 1; l < T; ++l) out[l] = Seg{S0.lvl_base[l], S0.lvl_len[l]};
+  if (T >= 1) out[T] = Seg{0, S0.lvl_len[T]};
+  return true;
+}
+
 // Split-K factor of a decode launch over the layer's current caches.
 static int pick_splits(balancekv_ctx* c, int layer) {
   const balancekv_config& f = c->cfg;
@@ -607,10 +625,12 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
   const int splits = pick_splits(c, layer);
   {
     ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
-    if (c->decode_maps)
-      BKV_CUDA(launch_decode_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                 static_cast<cudaStream_t>(stream)));
-    else
+    if (c->decode_maps) {
+      Seg hint[kMaxLevels + 1];
+      const bool alike = layer_seg_hint(c, layer, hint);
+      BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
+                                      nullptr, nullptr, 0, 0, 0, alike ? hint : nullptr, static_cast<cudaStream_t>(stream)));
+    } else
       BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
                              static_cast<cudaStream_t>(stream)));
   }
@@ -726,6 +746,8 @@ int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void
     }
     if (fits) {
       const int splits = pick_splits(c, layer);
+      Seg hint[kMaxLevels + 1];
+      const bool alike = layer_seg_hint(c, layer, hint);       // the table before this step's append
       const int rel = S0.start0 + S0.len0, idx0 = (int)S0.appended, new_len = S0.len0 + 1;
       for (int s : streams) {
         StreamState& S = c->st[s];
@@ -733,7 +755,8 @@ int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void
       }
       ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
       BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                      k_new, v_new, rel, idx0, new_len, static_cast<cudaStream_t>(stream)));
+                                      k_new, v_new, rel, idx0, new_len, alike ? hint : nullptr,
+                                      static_cast<cudaStream_t>(stream)));
       c->kernels_launched++;
       return BALANCEKV_OK;
     }

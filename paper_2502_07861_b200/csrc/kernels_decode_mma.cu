@@ -109,6 +109,10 @@ struct StepAppend {
   float* raw_acc;
   float* raw_ml;
   int keys_only;                // 1: only (M, sum) are wanted (a denominator instance): V is neither loaded nor multiplied
+  // Segment table of the layer's streams when they are all alike (the host mirrors it): saves the
+  // dependent global read at the start of a latency-bound launch.  n_seg = 0: read the table.
+  int n_seg;
+  Seg seg[kMaxLevels + 1];
 };
 
 struct TileRef {
@@ -164,7 +168,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid <= G.T) {
-    const Seg s = A.seg[(size_t)stream * (G.T + 1) + tid];
+    const Seg s = ap.n_seg ? ap.seg[tid] : A.seg[(size_t)stream * (G.T + 1) + tid];
     seg_s[tid] = s;
     lvl_tiles[tid] = (s.len + kTN - 1) / kTN;
   }
@@ -513,12 +517,12 @@ void decode_mma_release(void* maps) { delete static_cast<DecodeMaps*>(maps); }
 
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
 
 // Same scratch layout as launch_decode: ticket counters, then (stream, split, head) partial rows.
 cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                               int splits, int* status, const void* maps, cudaStream_t st) {
-  return launch_decode_step_mma(G, A, layer, q, out, scratch, splits, status, maps, nullptr, nullptr, 0, 0, 0, st);
+  return launch_decode_step_mma(G, A, layer, q, out, scratch, splits, status, maps, nullptr, nullptr, 0, 0, 0, nullptr, st);
 }
 
 // Un-normalised parts (see StepAppend::raw_acc) of the layer's streams for the two-instance estimator.
@@ -531,7 +535,7 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only};
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
                                                         tickets, status, ap, tm->k, tm->v);
   return cudaGetLastError();
@@ -575,15 +579,19 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
 // [B*H, d] bf16; all streams of the layer have the same level-0 fill).  k_new == nullptr: plain decode.
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, cudaStream_t st) {
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st) {
   if (!maps) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                      new_len, nullptr, nullptr, 0};
+  StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
+                new_len, nullptr, nullptr, 0, 0, {}};
+  if (seg_hint) {
+    ap.n_seg = G.T + 1;
+    for (int l = 0; l <= G.T; ++l) ap.seg[l] = seg_hint[l];
+  }
   // programmatic stream serialization: back-to-back decode steps overlap a launch with the
   // previous kernel's tail (see the kernel's prologue)
   cudaLaunchConfig_t cfg = {};
