@@ -439,18 +439,43 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   for (int i = tid; i < n_items; i += kThreads) {
     const int h = i / (kD / 4), c = (i % (kD / 4)) * 4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < splits; s += 8) {
-      float4 v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float4* src = reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c);
-        v[u] = s + u < splits ? (staged ? *src : __ldcg(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (staged) {
+      // partial rows in shared memory: plain shared loads, four independent accumulators
+      const float* base = sp_s + (size_t)h * PS + c;
+      const float* fac = cm + h;
+      float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+      int s = 0;
+      for (; s + 4 <= splits; s += 4) {
+        const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)(s + 0) * g * PS);
+        const float4 v1 = *reinterpret_cast<const float4*>(base + (size_t)(s + 1) * g * PS);
+        const float4 v2 = *reinterpret_cast<const float4*>(base + (size_t)(s + 2) * g * PS);
+        const float4 v3 = *reinterpret_cast<const float4*>(base + (size_t)(s + 3) * g * PS);
+        const float f0 = fac[(s + 0) * g], f1 = fac[(s + 1) * g], f2 = fac[(s + 2) * g], f3 = fac[(s + 3) * g];
+        a0.x = fmaf(v0.x, f0, a0.x); a0.y = fmaf(v0.y, f0, a0.y); a0.z = fmaf(v0.z, f0, a0.z); a0.w = fmaf(v0.w, f0, a0.w);
+        a1.x = fmaf(v1.x, f1, a1.x); a1.y = fmaf(v1.y, f1, a1.y); a1.z = fmaf(v1.z, f1, a1.z); a1.w = fmaf(v1.w, f1, a1.w);
+        a2.x = fmaf(v2.x, f2, a2.x); a2.y = fmaf(v2.y, f2, a2.y); a2.z = fmaf(v2.z, f2, a2.z); a2.w = fmaf(v2.w, f2, a2.w);
+        a3.x = fmaf(v3.x, f3, a3.x); a3.y = fmaf(v3.y, f3, a3.y); a3.z = fmaf(v3.z, f3, a3.z); a3.w = fmaf(v3.w, f3, a3.w);
       }
+      for (; s < splits; ++s) {
+        const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)s * g * PS);
+        const float f0 = fac[s * g];
+        a0.x = fmaf(v0.x, f0, a0.x); a0.y = fmaf(v0.y, f0, a0.y); a0.z = fmaf(v0.z, f0, a0.z); a0.w = fmaf(v0.w, f0, a0.w);
+      }
+      acc.x = (a0.x + a1.x) + (a2.x + a3.x); acc.y = (a0.y + a1.y) + (a2.y + a3.y);
+      acc.z = (a0.z + a1.z) + (a2.z + a3.z); acc.w = (a0.w + a1.w) + (a2.w + a3.w);
+    } else {
+      for (int s = 0; s < splits; s += 8) {
+        float4 v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float f = s + u < splits ? cm[(s + u) * g + h] : 0.f;
-        acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
-        acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+        for (int u = 0; u < 8; ++u)
+          v[u] = s + u < splits ? __ldcg(reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float f = s + u < splits ? cm[(s + u) * g + h] : 0.f;
+          acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
+          acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+        }
       }
     }
     if (ap.k_new) {
