@@ -295,7 +295,11 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     }
   }
   __syncthreads();
-  float* my_part = part + ((size_t)sl * splits + split) * g * PS;
+  // With a single split the CTA's partial is the stream's result: it stays in shared memory (behind
+  // the merge buffer) and the ticket, the fences and the staging copy are skipped.
+  constexpr uint32_t kSingleOff = 32768;
+  const bool single = splits == 1;
+  float* my_part = single ? reinterpret_cast<float*>(tiles + kSingleOff) : part + ((size_t)sl * splits + split) * g * PS;
   for (int i = tid; i < g * kD; i += kThreads) {
     const int h = i / kD, c = i % kD;
     float M = -INFINITY;
@@ -313,15 +317,19 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     if (c == 0) { my_part[h * PS + kD] = M; my_part[h * PS + kD + 1] = L; }
   }
   // ---- ticket: the last CTA of the stream combines the splits
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned old = atomicAdd(&tickets[sl], 1u);
-    is_last_s = old == (unsigned)(splits - 1);
+  if (!single) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const unsigned old = atomicAdd(&tickets[sl], 1u);
+      is_last_s = old == (unsigned)(splits - 1);
+    }
+    __syncthreads();
+    if (!is_last_s) return;
+    __threadfence();
+  } else {
+    __syncthreads();
   }
-  __syncthreads();
-  if (!is_last_s) return;
-  __threadfence();
   // Combine: first the (max, sum) pairs of all splits in one round of loads, then every thread
   // sums its output columns over the splits with independent loads.
   const float* sp = part + (size_t)sl * splits * g * PS;   // 16-byte aligned: rows of PS * 4 = 528 bytes
@@ -334,8 +342,8 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   // the idle tile ring (a single round trip); otherwise they are read from global memory.
   constexpr uint32_t kStageOff = 8192;                     // behind cm, cl, cM, cL, cN
   const uint32_t part_bytes = (uint32_t)splits * g * PS * sizeof(float);
-  const bool staged = part_bytes <= kStages * kStageBytes - kStageOff;
-  const float* sp_s = reinterpret_cast<const float*>(tiles + kStageOff);
+  const bool staged = single || part_bytes <= kStages * kStageBytes - kStageOff;
+  const float* sp_s = reinterpret_cast<const float*>(tiles + (single ? kSingleOff : kStageOff));
   if (ap.k_new) {
     // append (every CTA of the stream has taken its ticket, so nobody reads the old segment table
     // any more): one 256-byte row of K and of V, the position, the new length of C^0.  Done first,
@@ -386,7 +394,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     }
     if (tid < g * (kD / 4)) vn_pre = *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + (tid % (kD / 4)) * 4);
   }
-  if (staged) {
+  if (staged && !single) {
     if (tid == 0) {
       // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
       // (acquired above) come before the async-proxy copy
@@ -400,8 +408,8 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       if (tid == 0) { atomicCAS(status, kStatusOk, kStatusWaitTimeout); tickets[sl] = 0; }
       return;
     }
-    sp = sp_s;
   }
+  if (staged) sp = sp_s;
   for (int i = tid; i < splits * g; i += kThreads) {
     const float* rowp = sp + (size_t)i * PS;
     cm[i] = staged ? rowp[kD] : __ldcg(rowp + kD);
@@ -496,7 +504,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
     o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
   }
-  if (tid == 0) tickets[sl] = 0;   // ready for the next launch
+  if (tid == 0 && !single) tickets[sl] = 0;   // ready for the next launch
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
