@@ -96,6 +96,10 @@ class Harness:
         self.ctx.stream_append_layer(layer, to_device(K, self.dtype), to_device(V, self.dtype))
         self.events.append(("append", layer, K, V))
 
+    def append_stream(self, seq, layer, head, K, V):
+        self.ctx.stream_append(seq, layer, head, to_device(K, self.dtype), to_device(V, self.dtype))
+        self.events.append(("append_stream", seq, layer, head, K, V))
+
     def compress(self):
         self.ctx.compress()
         self.events.append(("compress",))
@@ -109,6 +113,9 @@ class Harness:
             if ev[0] == "append":
                 if ev[1] == layer:
                     o.append(ev[2][seq, head], ev[3][seq, head])
+            elif ev[0] == "append_stream":          # ("append_stream", seq, layer, head, K[n,d], V[n,d])
+                if ev[1:4] == (seq, layer, head):
+                    o.append(ev[4], ev[5])
             else:
                 o.compress()
         return o
