@@ -28,8 +28,6 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
                                    int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
-cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
-                              int splits, int* status, const void* maps, cudaStream_t st);
 }  // namespace bkv
 
 #define BKV_CUDA(expr)                                                                    \

@@ -552,13 +552,9 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
                                    int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
 
-// Same scratch layout as launch_decode: ticket counters, then (stream, split, head) partial rows.
-cudaError_t launch_decode_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
-                              int splits, int* status, const void* maps, cudaStream_t st) {
-  return launch_decode_step_mma(G, A, layer, q, out, scratch, splits, status, maps, nullptr, nullptr, 0, 0, 0, nullptr, st);
-}
-
-// Un-normalised parts (see StepAppend::raw_acc) of the layer's streams for the two-instance estimator.
+// Scratch layout of all launches (as for launch_decode): ticket counters, then (stream, split, head)
+// partial rows.
+// Un-normalised parts (see StepAppend::raw_acc) of the layer's streams, for decode merged over slots.
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
                                     float* scratch, int splits, int* status, const void* maps, int keys_only,
                                     cudaStream_t st) {
