@@ -42,21 +42,32 @@ template <bool kBf16>
 __device__ inline void copy_rows_norm(uint4* __restrict__ dK, const uint4* __restrict__ sK, uint4* __restrict__ dV,
                                       const uint4* __restrict__ sV, float2* __restrict__ nrm, int rows, int chunks) {
   const int total = rows * chunks;
-  for (int i0 = 0; i0 < total; i0 += blockDim.x) {      // whole warps take part in the shuffles
-    const int i = i0 + threadIdx.x;
-    float k2 = 0.f, v2 = 0.f;
-    if (i < total) {
-      const uint4 a = sK[i], b = sV[i];
-      dK[i] = a;
-      dV[i] = b;
-      k2 = sumsq16<kBf16>(a);
-      v2 = sumsq16<kBf16>(b);
+  // two rounds of loads are issued before the first is consumed (the copy is latency bound)
+  for (int i0 = 0; i0 < total; i0 += 2 * blockDim.x) {    // whole warps take part in the shuffles
+    uint4 a[2], b[2];
+    int idx[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      idx[u] = i0 + u * blockDim.x + threadIdx.x;
+      if (idx[u] < total) { a[u] = sK[idx[u]]; b[u] = sV[idx[u]]; }
     }
-    for (int o = chunks / 2; o > 0; o >>= 1) {
-      k2 += __shfl_xor_sync(0xffffffffu, k2, o);
-      v2 += __shfl_xor_sync(0xffffffffu, v2, o);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (i0 + u * (int)blockDim.x >= total) break;       // block-uniform
+      const int i = idx[u];
+      float k2 = 0.f, v2 = 0.f;
+      if (i < total) {
+        dK[i] = a[u];
+        dV[i] = b[u];
+        k2 = sumsq16<kBf16>(a[u]);
+        v2 = sumsq16<kBf16>(b[u]);
+      }
+      for (int o = chunks / 2; o > 0; o >>= 1) {
+        k2 += __shfl_xor_sync(0xffffffffu, k2, o);
+        v2 += __shfl_xor_sync(0xffffffffu, v2, o);
+      }
+      if (i < total && i % chunks == 0) nrm[i / chunks] = make_float2(k2, v2);
     }
-    if (i < total && i % chunks == 0) nrm[i / chunks] = make_float2(k2, v2);
   }
 }
 
