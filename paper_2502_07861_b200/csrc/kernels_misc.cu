@@ -42,17 +42,17 @@ template <bool kBf16>
 __device__ inline void copy_rows_norm(uint4* __restrict__ dK, const uint4* __restrict__ sK, uint4* __restrict__ dV,
                                       const uint4* __restrict__ sV, float2* __restrict__ nrm, int rows, int chunks) {
   const int total = rows * chunks;
-  // two rounds of loads are issued before the first is consumed (the copy is latency bound)
-  for (int i0 = 0; i0 < total; i0 += 2 * blockDim.x) {    // whole warps take part in the shuffles
-    uint4 a[2], b[2];
-    int idx[2];
+  // four rounds of loads are issued before the first is consumed (the copy is latency bound)
+  for (int i0 = 0; i0 < total; i0 += 4 * blockDim.x) {    // whole warps take part in the shuffles
+    uint4 a[4], b[4];
+    int idx[4];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < 4; ++u) {
       idx[u] = i0 + u * blockDim.x + threadIdx.x;
       if (idx[u] < total) { a[u] = sK[idx[u]]; b[u] = sV[idx[u]]; }
     }
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < 4; ++u) {
       if (i0 + u * (int)blockDim.x >= total) break;       // block-uniform
       const int i = idx[u];
       float k2 = 0.f, v2 = 0.f;
