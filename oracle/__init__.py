@@ -18,3 +18,4 @@ from .binding import (  # noqa: F401
     weighted_attention,
     weighted_sums,
 )
+from .bucketing import NO_BUCKET, BucketedOracle, value_bucket  # noqa: F401,E402
