@@ -221,6 +221,38 @@ int balancekv_decode_attn_two(balancekv_ctx* ctx, int layer_num, int layer_den, 
 int balancekv_decode_attn_merged(balancekv_ctx* ctx, const int32_t* layers_num, int n_num, const int32_t* layers_den,
                                  int n_den, const void* q, void* out, void* stream);
 
+/* Algorithm 1's bucketing of the stream by value norm and its erasure of small-norm buckets.
+ * Token j belongs to the bucket index i with 2^(i-1) < ||v_j||_2 <= 2^i (a norm that is an exact
+ * power of two satisfies Algorithm 1's printed condition for two indices; the smaller is taken).
+ * The caller dedicates n_buckets (1..8) consecutive layer slots to one model layer: slot
+ * layer0 + b is the instance MR-Numerator_i of bucket i = i_top - b, so i_top >= log2 of the
+ * largest value norm that will ever arrive.  The call routes every row of the block to its
+ * instance (appended to that instance's C^0 in stream order, exactly as balancekv_stream_append
+ * would; the stored original position is the position inside the instance's own stream),
+ * updates the running maximum v_max of the value norms, and erases (empties, for good) every
+ * instance with 2^i <= erase_ratio * v_max -- Algorithm 1 prints the factor
+ * eps/(2n) e^{-r^2/sqrt d}, the proof of Theorem 1.1 uses eps/sqrt n; pass either, or 0 for no
+ * erasure.  Rows that are dropped instead of stored: zero values, rows of an erased bucket, rows
+ * below the lowest slot's bucket.  balancekv_compress then runs MergeAndReduce on every
+ * instance with independent coins, and balancekv_decode_attn_merged over the slots (numerator)
+ * and a balancekv_stream_append_layer_keys slot (denominator) is Algorithm 1's output ratio.
+ *   K, V        [n_tokens, head_dim] of one stream (balancekv_stream_append_bucketed) or
+ *               [n_seqs, n_kv_heads, n_tokens, head_dim] (.._layer_bucketed); device, 16-byte aligned
+ *   token_slot  device, may be NULL: int8 per row in the layout of K without head_dim, the slot
+ *               offset b the row went to, -1 if it was dropped
+ *   counts_host host, may be NULL: per stream n_buckets + 1 numbers, the rows sent to each slot
+ *               and the rows dropped
+ * Norms are compared as fp32 squared norms.  The call SYNCHRONISES `stream` once (the per-bucket
+ * counts drive the host bookkeeping of Algorithm 3) and may allocate routing buffers when a block
+ * is larger than any before.  Errors: BALANCEKV_E_INVAL for bad arguments or a value norm above
+ * 2^i_top (nothing is appended then), BALANCEKV_E_NOMEM when an instance would overflow. */
+int balancekv_stream_append_bucketed(balancekv_ctx* ctx, int seq, int layer0, int n_buckets, int i_top, int kv_head,
+                                     const void* K_blk, const void* V_blk, int n_tokens, float erase_ratio,
+                                     int8_t* token_slot, int32_t* counts_host, void* stream);
+int balancekv_stream_append_layer_bucketed(balancekv_ctx* ctx, int layer0, int n_buckets, int i_top, const void* K,
+                                           const void* V, int n_tokens, float erase_ratio, int8_t* token_slot,
+                                           int32_t* counts_host, void* stream);
+
 /* Kernel timing for roofline reports.  While enabled, every launch of the kernel classes
  * below is bracketed by CUDA events on its launch stream (at most 8192 launches between two
  * reads; later ones are not recorded).  balancekv_profile_read synchronises the device and

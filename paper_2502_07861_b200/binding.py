@@ -23,7 +23,8 @@ EXPORTS = [
     "balancekv_stats", "balancekv_strerror", "balancekv_plan_calls", "balancekv_reset",
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
-    "balancekv_decode_attn_two", "balancekv_decode_attn_merged",
+    "balancekv_decode_attn_two", "balancekv_decode_attn_merged", "balancekv_stream_append_bucketed",
+    "balancekv_stream_append_layer_bucketed",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -91,6 +92,8 @@ def load():
     lib.balancekv_decode_attn_two.argtypes = [vp, ci, ci, vp, vp, vp]
     lib.balancekv_decode_attn_merged.argtypes = [vp, vp, ci, vp, ci, vp, vp, vp]
     lib.balancekv_profile_read.argtypes = [vp, vp]
+    lib.balancekv_stream_append_bucketed.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
+    lib.balancekv_stream_append_layer_bucketed.argtypes = [vp, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     for name in EXPORTS:
         if name != "balancekv_strerror":
@@ -220,6 +223,39 @@ class Context:
         """Denominator instance of Algorithm 1: append (k_j, 1); K [B, H, n, d] on the device."""
         _check(self.lib.balancekv_stream_append_layer_keys(self._h, layer, self._dev(K, "K"), K.shape[2],
                                                            _stream_ptr(stream)), "balancekv_stream_append_layer_keys")
+
+    def stream_append_layer_bucketed(self, layer0, n_buckets, i_top, K, V, erase_ratio=0.0, want_slots=False,
+                                     stream=None):
+        """Algorithm 1's bucketing step for every stream of a layer: K, V [B, H, n, d] on the device;
+        slot layer0 + b receives the rows with 2^(i_top-b-1) < ||v|| <= 2^(i_top-b).  Returns the
+        per-stream counts [B*H, n_buckets + 1] (last column: dropped rows) and, if asked, the int8
+        slot of every row [B, H, n]."""
+        import numpy as np
+        import torch
+
+        assert K.shape == V.shape and K.dim() == 4
+        counts = np.zeros((K.shape[0] * K.shape[1], n_buckets + 1), np.int32)
+        slots = torch.empty(K.shape[:3], dtype=torch.int8, device=K.device) if want_slots else None
+        _check(self.lib.balancekv_stream_append_layer_bucketed(
+            self._h, layer0, n_buckets, i_top, self._dev(K, "K"), self._dev(V, "V"), K.shape[2], float(erase_ratio),
+            slots.data_ptr() if want_slots else None, counts.ctypes.data, _stream_ptr(stream)),
+            "balancekv_stream_append_layer_bucketed")
+        return (counts, slots) if want_slots else counts
+
+    def stream_append_bucketed(self, seq, layer0, n_buckets, i_top, kv_head, K, V, erase_ratio=0.0, want_slots=False,
+                               stream=None):
+        """Same for one stream: K, V [n, d] on the device."""
+        import numpy as np
+        import torch
+
+        assert K.shape == V.shape and K.dim() == 2
+        counts = np.zeros((1, n_buckets + 1), np.int32)
+        slots = torch.empty(K.shape[0], dtype=torch.int8, device=K.device) if want_slots else None
+        _check(self.lib.balancekv_stream_append_bucketed(
+            self._h, seq, layer0, n_buckets, i_top, kv_head, self._dev(K, "K"), self._dev(V, "V"), K.shape[0],
+            float(erase_ratio), slots.data_ptr() if want_slots else None, counts.ctypes.data, _stream_ptr(stream)),
+            "balancekv_stream_append_bucketed")
+        return (counts[0], slots) if want_slots else counts[0]
 
     def decode_attn_two(self, layer_num, layer_den, q, out=None, stream=None):
         """Algorithm 1's output ratio: numerator from slot layer_num, denominator from slot layer_den."""

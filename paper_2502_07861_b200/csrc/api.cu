@@ -1,10 +1,13 @@
 // C ABI of the BalanceKV library: context, memory layout, launch scheduling.
 // Every step of the hot path runs in the CUDA kernels of this directory; this file only
 // validates arguments, keeps Algorithm 3's bookkeeping (sched.h) and enqueues launches.
+#include <climits>
 #include <cmath>
+#include <cstdint>
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "../../include/balancekv.h"
@@ -109,6 +112,19 @@ struct balancekv_ctx {
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
   std::vector<std::vector<int>> layer_stream_ids;
+
+  // value-norm buckets (Algorithm 1): running v_max^2 and the largest erased bucket index, indexed
+  // by the stream of the first bucket slot; routing buffers sized for the largest block so far
+  std::vector<float> bucket_vmax2;
+  std::vector<int32_t> bucket_erase_max;
+  float* bkt_ns = nullptr;
+  int8_t* bkt_slot = nullptr;
+  int32_t* bkt_rank = nullptr;
+  unsigned* bkt_vmax_bits = nullptr;
+  BucketOut* bkt_out = nullptr;
+  BucketOut* bkt_out_host = nullptr;    // pinned
+  size_t bkt_rows = 0, bkt_streams = 0;
+  int64_t bucket_dropped = 0;
 
   // optional per-class kernel timing
   unsigned profiling = 0;                   // bit per kernel class
@@ -346,6 +362,10 @@ int balancekv_destroy(balancekv_ctx* c) {
                   c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->unit_V};
   for (void* p : ptrs)
     if (p) cudaFree(p);
+  void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out};
+  for (void* p : bkt)
+    if (p) cudaFree(p);
+  if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
   if (c->h_ring) cudaFreeHost(c->h_ring);
   if (c->step_host) cudaFreeHost(c->step_host);
   for (cudaEvent_t e : c->step_ev)
@@ -901,10 +921,145 @@ int balancekv_debug_call(balancekv_ctx* c, int seq, int layer, int kv_head, int 
   return BALANCEKV_OK;
 }
 
+// Algorithm 1's bucketing step for the streams `heads` (pairs seq, kv_head) whose blocks lie
+// consecutively in K, V.  Slot layer0 + b is the instance of bucket index i_top - b.
+static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<int, int>>& heads, int layer0,
+                                int n_buckets, int i_top, const void* K, const void* V, int n, float rho,
+                                int8_t* token_slot, int32_t* counts_host, cudaStream_t st) {
+  const balancekv_config& f = c->cfg;
+  const Layout& Lo = c->Lo;
+  if (!K || !V || n < 1 || n > (1 << 22) || !aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
+  if (n_buckets < 1 || n_buckets > kMaxBuckets || layer0 < 0 || layer0 + n_buckets > f.n_layers) return BALANCEKV_E_INVAL;
+  if (i_top < -60 || i_top > 60 || !(rho >= 0.f) || rho > 1.f) return BALANCEKV_E_INVAL;
+  const int n_sl = (int)heads.size();
+  if (n_sl < 1) return BALANCEKV_E_INVAL;
+  if (c->bucket_vmax2.empty()) {
+    c->bucket_vmax2.assign(c->n_streams, 0.f);
+    c->bucket_erase_max.assign(c->n_streams, INT32_MIN);
+  }
+  // routing buffers (grown with the largest block; the call synchronises the stream anyway)
+  if ((size_t)n_sl * n > c->bkt_rows || (size_t)n_sl > c->bkt_streams) {
+    BKV_CUDA(cudaStreamSynchronize(st));
+    void* old[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out};
+    for (void* p : old)
+      if (p) cudaFree(p);
+    if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
+    c->bkt_ns = nullptr; c->bkt_slot = nullptr; c->bkt_rank = nullptr; c->bkt_vmax_bits = nullptr; c->bkt_out = nullptr;
+    c->bkt_out_host = nullptr;
+    c->bkt_rows = std::max(c->bkt_rows, (size_t)n_sl * n);
+    c->bkt_streams = std::max(c->bkt_streams, (size_t)n_sl);
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_ns), sizeof(float) * c->bkt_rows));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_slot), c->bkt_rows));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_rank), sizeof(int32_t) * c->bkt_rows));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_vmax_bits), sizeof(unsigned) * c->bkt_streams));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_out), sizeof(BucketOut) * c->bkt_streams));
+    BKV_CUDA(cudaMallocHost(reinterpret_cast<void**>(&c->bkt_out_host), sizeof(BucketOut) * c->bkt_streams));
+  }
+  std::vector<BucketIn> in(n_sl);
+  for (int i = 0; i < n_sl; ++i) {
+    const int s0 = stream_id(c, heads[i].first, layer0, heads[i].second);
+    in[i].prev_vmax2 = c->bucket_vmax2[s0];
+    in[i].prev_erase_max = c->bucket_erase_max[s0];
+  }
+  void* d_in = nullptr;
+  int rc = ring_push(c, in.data(), in.size() * sizeof(BucketIn), st, &d_in);
+  if (rc) return rc;
+  {
+    ProfScope ps(c, 0, st);
+    BKV_CUDA(launch_bucket_route(c->G, V, n_sl, n, n_buckets, i_top, rho * rho, static_cast<const BucketIn*>(d_in),
+                                 c->bkt_vmax_bits, c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_out, st));
+  }
+  c->kernels_launched += 2;
+  BKV_CUDA(cudaMemcpyAsync(c->bkt_out_host, c->bkt_out, sizeof(BucketOut) * n_sl, cudaMemcpyDeviceToHost, st));
+  BKV_CUDA(cudaStreamSynchronize(st));   // the counts decide the host bookkeeping of every instance
+  const BucketOut* out = c->bkt_out_host;
+  const int T = Lo.T;
+  const int max_pending = T == 0 ? f.max_tokens : (f.max_pending > 0 ? std::min(f.max_pending, f.max_tokens) : f.max_tokens);
+  for (int i = 0; i < n_sl; ++i) {
+    if (out[i].above > 0) return BALANCEKV_E_INVAL;        // a value norm above 2^i_top: nothing was appended
+    for (int b = 0; b < n_buckets; ++b) {
+      const StreamState& S = c->st[stream_id(c, heads[i].first, layer0 + b, heads[i].second)];
+      const int m = out[i].count[b];
+      if (S.appended + m > f.max_tokens || S.pending + m > max_pending) return BALANCEKV_E_NOMEM;
+      if ((int64_t)S.start0 + S.len0 + m > Lo.cap0) return BALANCEKV_E_NOMEM;
+    }
+  }
+  std::vector<BucketDst> dst((size_t)n_sl * n_buckets);
+  for (int i = 0; i < n_sl; ++i) {
+    const int s0 = stream_id(c, heads[i].first, layer0, heads[i].second);
+    c->bucket_vmax2[s0] = out[i].vmax2;
+    c->bucket_erase_max[s0] = out[i].erase_max;
+    c->bucket_dropped += out[i].dropped;
+    for (int b = 0; b < n_buckets; ++b) {
+      const int s = stream_id(c, heads[i].first, layer0 + b, heads[i].second);
+      StreamState& S = c->st[s];
+      BucketDst& D = dst[(size_t)i * n_buckets + b];
+      D.pad = 0;
+      if (i_top - b <= out[i].erase_max) {
+        // "erase all MR-Numerator_i with 2^i <= rho * v_max": the instance forgets its sets
+        if (S.appended > 0) {
+          c->bucket_dropped += S.appended;
+          S = StreamState();
+          BKV_CUDA(cudaMemsetAsync(c->A.seg + (size_t)s * (T + 1), 0, sizeof(Seg) * (T + 1), st));
+        }
+        D.dst_row = 0; D.idx0 = 0; D.stream = -1; D.new_len = 0;
+        continue;
+      }
+      const int m = out[i].count[b];
+      D.dst_row = (int64_t)s * Lo.R + Lo.region_off[0] + S.start0 + S.len0;
+      D.idx0 = (int32_t)S.appended;
+      D.stream = m > 0 ? s : -1;
+      S.len0 += m; S.appended += m; S.pending += m;
+      D.new_len = S.len0;
+      c->tokens_appended += m;
+    }
+  }
+  void* d_dst = nullptr;
+  rc = ring_push(c, dst.data(), dst.size() * sizeof(BucketDst), st, &d_dst);
+  if (rc) return rc;
+  {
+    ProfScope ps(c, 0, st);
+    BKV_CUDA(launch_bucket_scatter(c->G, c->A, K, V, n_sl, n, n_buckets, c->bkt_slot, c->bkt_rank, c->bkt_ns,
+                                   static_cast<const BucketDst*>(d_dst), st));
+  }
+  c->kernels_launched++;
+  if (token_slot)
+    BKV_CUDA(cudaMemcpyAsync(token_slot, c->bkt_slot, (size_t)n_sl * n, cudaMemcpyDeviceToDevice, st));
+  if (counts_host)
+    for (int i = 0; i < n_sl; ++i) {
+      int32_t* row = counts_host + (size_t)i * (n_buckets + 1);
+      for (int b = 0; b < n_buckets; ++b) row[b] = out[i].count[b];
+      row[n_buckets] = out[i].dropped;
+    }
+  return BALANCEKV_OK;
+}
+
+int balancekv_stream_append_bucketed(balancekv_ctx* c, int seq, int layer0, int n_buckets, int i_top, int kv_head,
+                                     const void* K_blk, const void* V_blk, int n_tokens, float erase_ratio,
+                                     int8_t* token_slot, int32_t* counts_host, void* stream) {
+  if (!c || seq < 0 || seq >= c->cfg.n_seqs || kv_head < 0 || kv_head >= c->cfg.n_kv_heads) return BALANCEKV_E_INVAL;
+  std::vector<std::pair<int, int>> heads{{seq, kv_head}};
+  return append_bucketed_impl(c, heads, layer0, n_buckets, i_top, K_blk, V_blk, n_tokens, erase_ratio, token_slot,
+                              counts_host, static_cast<cudaStream_t>(stream));
+}
+
+int balancekv_stream_append_layer_bucketed(balancekv_ctx* c, int layer0, int n_buckets, int i_top, const void* K,
+                                           const void* V, int n_tokens, float erase_ratio, int8_t* token_slot,
+                                           int32_t* counts_host, void* stream) {
+  if (!c) return BALANCEKV_E_INVAL;
+  std::vector<std::pair<int, int>> heads;
+  for (int s = 0; s < c->cfg.n_seqs; ++s)
+    for (int h = 0; h < c->cfg.n_kv_heads; ++h) heads.push_back({s, h});
+  return append_bucketed_impl(c, heads, layer0, n_buckets, i_top, K, V, n_tokens, erase_ratio, token_slot, counts_host,
+                              static_cast<cudaStream_t>(stream));
+}
+
 int balancekv_reset(balancekv_ctx* c, void* stream) {
   if (!c) return BALANCEKV_E_INVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   for (StreamState& S : c->st) S = StreamState();
+  c->bucket_vmax2.clear();
+  c->bucket_erase_max.clear();
   BKV_CUDA(cudaMemsetAsync(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (c->cfg.levels + 1), st));
   return BALANCEKV_OK;
 }

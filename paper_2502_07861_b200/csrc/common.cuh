@@ -31,6 +31,28 @@ struct AppendDesc {
   int32_t pad;
 };
 
+// Value-norm buckets (Algorithm 1): per-stream input and result of the routing pass, and the
+// destination of one (stream, bucket) pair in the arena.
+constexpr int kMaxBuckets = 8;
+struct BucketIn {
+  float prev_vmax2;        // v_max^2 over the stream's earlier blocks
+  int32_t prev_erase_max;  // largest bucket index erased so far (INT32_MIN: none)
+};
+struct BucketOut {
+  int32_t count[kMaxBuckets];  // tokens of the block per slot
+  int32_t dropped;             // zero values, erased buckets, indices below the lowest slot
+  int32_t above;               // tokens above the highest slot (the block is then refused)
+  int32_t erase_max;           // largest erased bucket index after the block
+  float vmax2;                 // v_max^2 after the block
+};
+struct BucketDst {
+  int64_t dst_row;    // arena row that receives the slot's first token of the block
+  int32_t idx0;       // that token's position in the instance's stream
+  int32_t stream;     // instance's stream (segment table row); -1: nothing to update
+  int32_t new_len;    // level-0 length after the block
+  int32_t pad;
+};
+
 // One move of a stream's level-0 remainder to the front of its region.
 struct MoveDesc {
   int64_t src_row, dst_row;
@@ -116,6 +138,11 @@ __device__ inline float warp_sum(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+__device__ inline int warp_sum_int(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
 __device__ inline float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -156,6 +183,12 @@ cudaError_t launch_decode(const Geom& G, const Arena& A, int layer, const void* 
                           int splits, int* status, cudaStream_t st);
 cudaError_t launch_fill_weights(float* w, int n, float value, cudaStream_t st);
 cudaError_t launch_seg_update(const Arena& A, const SegUpdate* ups, int n, cudaStream_t st);
+cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, int n_buckets, int i_top, float rho2,
+                                const BucketIn* in, unsigned* vmax2_bits, float* ns, int8_t* slot, int32_t* rank,
+                                BucketOut* out, cudaStream_t st);
+cudaError_t launch_bucket_scatter(const Geom& G, const Arena& A, const void* K, const void* V, int n_sl, int n,
+                                  int n_buckets, const int8_t* slot, const int32_t* rank, const float* ns,
+                                  const BucketDst* dst, cudaStream_t st);
 int walk_simt_supported(int d);
 size_t walk_simt_smem_bytes(int d, int t);
 
