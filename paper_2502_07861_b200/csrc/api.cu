@@ -121,6 +121,8 @@ struct balancekv_ctx {
   int8_t* bkt_slot = nullptr;
   int32_t* bkt_rank = nullptr;
   unsigned* bkt_vmax_bits = nullptr;
+  int32_t* bkt_chunk_cnt = nullptr;     // per (stream, chunk of the block): counts, then their prefix
+  size_t bkt_chunk_ints = 0;
   BucketOut* bkt_out = nullptr;
   BucketOut* bkt_out_host = nullptr;    // pinned
   size_t bkt_rows = 0, bkt_streams = 0;
@@ -362,7 +364,7 @@ int balancekv_destroy(balancekv_ctx* c) {
                   c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->unit_V};
   for (void* p : ptrs)
     if (p) cudaFree(p);
-  void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out};
+  void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out, c->bkt_chunk_cnt};
   for (void* p : bkt)
     if (p) cudaFree(p);
   if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
@@ -938,14 +940,16 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
     c->bucket_erase_max.assign(c->n_streams, INT32_MIN);
   }
   // routing buffers (grown with the largest block; the call synchronises the stream anyway)
-  if ((size_t)n_sl * n > c->bkt_rows || (size_t)n_sl > c->bkt_streams) {
+  if ((size_t)n_sl * n > c->bkt_rows || (size_t)n_sl > c->bkt_streams || bucket_chunk_count_ints(n_sl, n) > c->bkt_chunk_ints) {
     BKV_CUDA(cudaStreamSynchronize(st));
-    void* old[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out};
+    void* old[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out, c->bkt_chunk_cnt};
     for (void* p : old)
       if (p) cudaFree(p);
     if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
     c->bkt_ns = nullptr; c->bkt_slot = nullptr; c->bkt_rank = nullptr; c->bkt_vmax_bits = nullptr; c->bkt_out = nullptr;
-    c->bkt_out_host = nullptr;
+    c->bkt_out_host = nullptr; c->bkt_chunk_cnt = nullptr;
+    c->bkt_chunk_ints = std::max(c->bkt_chunk_ints, bucket_chunk_count_ints(n_sl, n));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_chunk_cnt), sizeof(int32_t) * c->bkt_chunk_ints));
     c->bkt_rows = std::max(c->bkt_rows, (size_t)n_sl * n);
     c->bkt_streams = std::max(c->bkt_streams, (size_t)n_sl);
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->bkt_ns), sizeof(float) * c->bkt_rows));
@@ -967,9 +971,9 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
   {
     ProfScope ps(c, 0, st);
     BKV_CUDA(launch_bucket_route(c->G, V, n_sl, n, n_buckets, i_top, rho * rho, static_cast<const BucketIn*>(d_in),
-                                 c->bkt_vmax_bits, c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_out, st));
+                                 c->bkt_vmax_bits, c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_chunk_cnt, c->bkt_out, st));
   }
-  c->kernels_launched += 2;
+  c->kernels_launched += 3;
   BKV_CUDA(cudaMemcpyAsync(c->bkt_out_host, c->bkt_out, sizeof(BucketOut) * n_sl, cudaMemcpyDeviceToHost, st));
   BKV_CUDA(cudaStreamSynchronize(st));   // the counts decide the host bookkeeping of every instance
   const BucketOut* out = c->bkt_out_host;
@@ -1019,8 +1023,8 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
   if (rc) return rc;
   {
     ProfScope ps(c, 0, st);
-    BKV_CUDA(launch_bucket_scatter(c->G, c->A, K, V, n_sl, n, n_buckets, c->bkt_slot, c->bkt_rank, c->bkt_ns,
-                                   static_cast<const BucketDst*>(d_dst), st));
+    BKV_CUDA(launch_bucket_scatter(c->G, c->A, K, V, n_sl, n, n_buckets, c->bkt_slot, c->bkt_rank, c->bkt_chunk_cnt,
+                                   c->bkt_ns, static_cast<const BucketDst*>(d_dst), st));
   }
   c->kernels_launched++;
   if (token_slot)

@@ -183,12 +183,14 @@ cudaError_t launch_decode(const Geom& G, const Arena& A, int layer, const void* 
                           int splits, int* status, cudaStream_t st);
 cudaError_t launch_fill_weights(float* w, int n, float value, cudaStream_t st);
 cudaError_t launch_seg_update(const Arena& A, const SegUpdate* ups, int n, cudaStream_t st);
+int bucket_scan_chunks(int n);
+size_t bucket_chunk_count_ints(int n_sl, int n);   // ints of the per-chunk count table of the routing pass
 cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, int n_buckets, int i_top, float rho2,
                                 const BucketIn* in, unsigned* vmax2_bits, float* ns, int8_t* slot, int32_t* rank,
-                                BucketOut* out, cudaStream_t st);
+                                int32_t* chunk_cnt, BucketOut* out, cudaStream_t st);
 cudaError_t launch_bucket_scatter(const Geom& G, const Arena& A, const void* K, const void* V, int n_sl, int n,
-                                  int n_buckets, const int8_t* slot, const int32_t* rank, const float* ns,
-                                  const BucketDst* dst, cudaStream_t st);
+                                  int n_buckets, const int8_t* slot, const int32_t* rank, const int32_t* chunk_base,
+                                  const float* ns, const BucketDst* dst, cudaStream_t st);
 int walk_simt_supported(int d);
 size_t walk_simt_smem_bytes(int d, int t);
 

@@ -1,8 +1,9 @@
 // Value-norm buckets of BalanceKV (Algorithm 1, the bucketing step and the erasure of small-norm
 // buckets): token j goes to the MergeAndReduce instance of the index i with 2^(i-1) < ||v_j|| <= 2^i,
-// instances whose bucket satisfies 2^i <= rho * v_max are erased.  Three kernels: squared value
-// norms + running maximum, a stable partition of the block's tokens by bucket (one CTA per
-// stream), and the copy of every kept row into the level-0 set of its bucket's instance.
+// instances whose bucket satisfies 2^i <= rho * v_max are erased.  Four kernels: squared value
+// norms + running maximum; a stable partition of the block's tokens by bucket in two parts (ranks
+// inside chunks of 2048 tokens, then the prefix over a stream's chunks); and the copy of every
+// kept row into the level-0 set of its bucket's instance.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -14,7 +15,9 @@ namespace bkv {
 
 namespace {
 
-constexpr int kScanThreads = 1024;
+constexpr int kScanThreads = 256;
+constexpr int kScanChunk = 2048;               // tokens per CTA of the partition's first part
+constexpr int kCountCols = kMaxBuckets + 2;    // per-slot counts, dropped, above
 constexpr int kRowsPerBlock = 64;
 
 template <bool kBf16>
@@ -37,20 +40,31 @@ __device__ inline float sumsq_piece(const uint4& v) {
 }
 
 // ||v_j||^2 of every row of the block (chunks = 16-byte pieces of a row: 8, 16 or 32 lanes share
-// a row) and the maximum per stream.  grid (row groups, streams), 256 threads.
+// a row) and the maximum per stream.  grid (row groups, streams), 256 threads; a thread's loads of
+// all passes are issued before the first is reduced.
 template <bool kBf16>
 __global__ void __launch_bounds__(256)
 bucket_norms_kernel(const void* __restrict__ V, int n, int chunks, float* __restrict__ ns, unsigned* __restrict__ vmax2_bits) {
   const int sl = blockIdx.y;
-  const int rows_per_pass = blockDim.x / chunks;
+  const int rows_per_pass = blockDim.x / chunks;         // 32, 16 or 8
   const int row_in = threadIdx.x / chunks, piece = threadIdx.x % chunks;
   const uint4* src = reinterpret_cast<const uint4*>(V) + (size_t)sl * n * chunks;
+  const int row0 = blockIdx.x * kRowsPerBlock;
+  const int row_end = min(n, row0 + kRowsPerBlock);
+  constexpr int kMaxPasses = kRowsPerBlock / 8;
+  uint4 v[kMaxPasses];
+#pragma unroll
+  for (int u = 0; u < kMaxPasses; ++u) {
+    const int r = row0 + u * rows_per_pass + row_in;
+    v[u] = make_uint4(0u, 0u, 0u, 0u);
+    if (u * rows_per_pass < kRowsPerBlock && r < row_end) v[u] = src[(size_t)r * chunks + piece];
+  }
   float mx = 0.f;
-  const int row_end = min(n, (int)(blockIdx.x + 1) * kRowsPerBlock);
-  for (int r0 = blockIdx.x * kRowsPerBlock; r0 < row_end; r0 += rows_per_pass) {
-    const int r = r0 + row_in;
-    float s = 0.f;
-    if (r < row_end) s = sumsq_piece<kBf16>(src[(size_t)r * chunks + piece]);
+#pragma unroll
+  for (int u = 0; u < kMaxPasses; ++u) {
+    if (u * rows_per_pass >= kRowsPerBlock) break;       // block-uniform
+    const int r = row0 + u * rows_per_pass + row_in;
+    float s = sumsq_piece<kBf16>(v[u]);
     for (int o = chunks / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (r < row_end && piece == 0) ns[(size_t)sl * n + r] = s;
     mx = fmaxf(mx, s);
@@ -68,18 +82,9 @@ __device__ inline int bucket_of(float ns) {
   return (a + 1) >> 1;                       // ceil(a / 2), also for negative a
 }
 
-// Stable partition of a stream's block by bucket.  One CTA per stream; thread x owns the
-// contiguous tokens [x*per, (x+1)*per).  Writes, per token, its slot (or -1) and its rank among
-// the block's tokens of the same slot; per stream, the counts and the erase decision.
-__global__ void __launch_bounds__(kScanThreads)
-bucket_scan_kernel(const float* __restrict__ ns, int n, int n_buckets, int i_top, float rho2,
-                   const BucketIn* __restrict__ in, const unsigned* __restrict__ vmax2_bits, int8_t* __restrict__ slot,
-                   int32_t* __restrict__ rank, BucketOut* __restrict__ out) {
-  __shared__ int warp_tot[kMaxBuckets][kScanThreads / 32];
-  __shared__ int tot[kMaxBuckets];
-  const int sl = blockIdx.x;
-  const float vmax2 = fmaxf(in[sl].prev_vmax2, __uint_as_float(vmax2_bits[sl]));
-  // largest erased index: 4^i <= rho^2 * v_max^2
+// The largest erased bucket index after the block: 4^i <= rho^2 * v_max^2 (INT32_MIN: none).
+__device__ inline int erase_index(float rho2, const BucketIn& in, unsigned vmax2_bits) {
+  const float vmax2 = fmaxf(in.prev_vmax2, __uint_as_float(vmax2_bits));
   int erase_max = INT32_MIN;
   const float thr = rho2 * vmax2;
   if (thr > 0.f) {
@@ -87,76 +92,107 @@ bucket_scan_kernel(const float* __restrict__ ns, int n, int n_buckets, int i_top
     frexpf(thr, &e);                         // log2(thr) in [e-1, e)
     erase_max = (e - 1) >> 1;                // floor((e-1)/2)
   }
-  erase_max = max(erase_max, in[sl].prev_erase_max);
-  const int per = (n + kScanThreads - 1) / kScanThreads;
-  const int j0 = min(n, (int)threadIdx.x * per), j1 = min(n, j0 + per);
-  const float* x = ns + (size_t)sl * n;
-  int cnt[kMaxBuckets];
-#pragma unroll
-  for (int b = 0; b < kMaxBuckets; ++b) cnt[b] = 0;
-  int dropped = 0, above = 0;
-  for (int j = j0; j < j1; ++j) {
-    const float v = x[j];
-    int b = -1;
-    if (v > 0.f) {
-      const int i = bucket_of(v);
-      if (i > i_top) ++above;
-      else if (i > erase_max && i_top - i < n_buckets) b = i_top - i;
-    }
-    if (b < 0) ++dropped;
-#pragma unroll
-    for (int bb = 0; bb < kMaxBuckets; ++bb) cnt[bb] += (bb == b);
-    slot[(size_t)sl * n + j] = (int8_t)b;
-  }
-  // exclusive prefix of the per-thread counts, bucket by bucket
+  return max(erase_max, in.prev_erase_max);
+}
+
+// Stable partition of a stream's block by bucket, first part.  grid (chunks of kScanChunk tokens,
+// streams), 256 threads; warp w owns the contiguous tokens [w*256, (w+1)*256) of the chunk and
+// walks them 32 at a time (ballots give the rank among equal slots).  Writes, per token, its slot
+// (or -1) and its rank among the chunk's tokens of the same slot; per chunk, the counts.
+__global__ void __launch_bounds__(kScanThreads)
+bucket_scan_kernel(const float* __restrict__ ns, int n, int n_chunks, int n_buckets, int i_top, float rho2,
+                   const BucketIn* __restrict__ in, const unsigned* __restrict__ vmax2_bits, int8_t* __restrict__ slot,
+                   int32_t* __restrict__ rank, int32_t* __restrict__ chunk_cnt) {
+  constexpr int kWarps = kScanThreads / 32, kRounds = kScanChunk / kScanThreads;
+  __shared__ int warp_tot[kCountCols][kWarps];
+  const int sl = blockIdx.y, chunk = blockIdx.x;
+  const int erase_max = erase_index(rho2, in[sl], vmax2_bits[sl]);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int excl[kMaxBuckets];
+  const unsigned lt = (1u << lane) - 1u;
+  const size_t base = (size_t)sl * n;
+  const int j0 = chunk * kScanChunk + warp * (kScanChunk / kWarps);
+  float x[kRounds];
 #pragma unroll
-  for (int b = 0; b < kMaxBuckets; ++b) {
-    int v = cnt[b];
+  for (int u = 0; u < kRounds; ++u) {
+    const int j = j0 + u * 32 + lane;
+    x[u] = j < n ? ns[base + j] : -1.f;
+  }
+  int run[kCountCols];                                   // warp-uniform running counts: slots, dropped, above
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int u = __shfl_up_sync(0xffffffffu, v, o);
-      if (lane >= o) v += u;
+  for (int b = 0; b < kCountCols; ++b) run[b] = 0;
+  int my_slot[kRounds], my_rank[kRounds];
+#pragma unroll
+  for (int u = 0; u < kRounds; ++u) {
+    int b = -3;                                          // past the end of the block
+    if (x[u] >= 0.f) {
+      b = kMaxBuckets;                                   // dropped
+      if (x[u] > 0.f) {
+        const int i = bucket_of(x[u]);
+        if (i > i_top) b = kMaxBuckets + 1;              // above the highest slot
+        else if (i > erase_max && i_top - i < n_buckets) b = i_top - i;
+      }
     }
-    excl[b] = v - cnt[b];
-    if (lane == 31) warp_tot[b][warp] = v;
-  }
-  __syncthreads();
-  if (warp < kMaxBuckets) {
-    int v = warp_tot[warp][lane];
-    const int own = v;
+    my_slot[u] = b;
+    my_rank[u] = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int u = __shfl_up_sync(0xffffffffu, v, o);
-      if (lane >= o) v += u;
+    for (int bb = 0; bb < kCountCols; ++bb) {
+      const unsigned m = __ballot_sync(0xffffffffu, b == bb);
+      if (b == bb) my_rank[u] = run[bb] + __popc(m & lt);
+      run[bb] += __popc(m);
     }
-    warp_tot[warp][lane] = v - own;
-    if (lane == 31) tot[warp] = v;
   }
-  __syncthreads();
-#pragma unroll
-  for (int b = 0; b < kMaxBuckets; ++b) excl[b] += warp_tot[b][warp];
-  for (int j = j0; j < j1; ++j) {
-    const int b = slot[(size_t)sl * n + j];
-    int r = 0;
-#pragma unroll
-    for (int bb = 0; bb < kMaxBuckets; ++bb)
-      if (bb == b) r = excl[bb]++;
-    rank[(size_t)sl * n + j] = r;
-  }
-  dropped = warp_sum_int(dropped);
-  above = warp_sum_int(above);
-  if (threadIdx.x == 0) { out[sl].dropped = 0; out[sl].above = 0; }
-  __syncthreads();
   if (lane == 0) {
-    if (dropped) atomicAdd(&out[sl].dropped, dropped);
-    if (above) atomicAdd(&out[sl].above, above);
+#pragma unroll
+    for (int bb = 0; bb < kCountCols; ++bb) warp_tot[bb][warp] = run[bb];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < kRounds; ++u) {
+    const int j = j0 + u * 32 + lane;
+    const int b = my_slot[u];
+    if (j < n) {
+      int off = 0;
+      if (b >= 0 && b < kMaxBuckets)
+        for (int w = 0; w < warp; ++w) off += warp_tot[b][w];
+      slot[base + j] = (int8_t)(b < kMaxBuckets ? b : -1);
+      rank[base + j] = off + my_rank[u];
+    }
+  }
+  if (threadIdx.x < kCountCols) {
+    int t = 0;
+    for (int w = 0; w < kWarps; ++w) t += warp_tot[threadIdx.x][w];
+    chunk_cnt[((size_t)sl * n_chunks + chunk) * kCountCols + threadIdx.x] = t;
+  }
+}
+
+// Second part: per stream, the exclusive prefix of the chunks' counts (in place) and the totals.
+// grid (streams), kCountCols warps: warp b scans column b, 32 chunks at a time.
+__global__ void __launch_bounds__(kCountCols * 32)
+bucket_prefix_kernel(int n_chunks, float rho2, const BucketIn* __restrict__ in, const unsigned* __restrict__ vmax2_bits,
+                     int32_t* __restrict__ chunk_cnt, BucketOut* __restrict__ out) {
+  const int sl = blockIdx.x, col = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int32_t* c = chunk_cnt + (size_t)sl * n_chunks * kCountCols + col;
+  int carry = 0;
+  for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+    const int i = c0 + lane;
+    const int own = i < n_chunks ? c[(size_t)i * kCountCols] : 0;
+    int v = own;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += u;
+    }
+    if (i < n_chunks) c[(size_t)i * kCountCols] = carry + v - own;
+    carry += __shfl_sync(0xffffffffu, v, 31);
+  }
+  if (lane == 0) {
+    if (col < kMaxBuckets) out[sl].count[col] = carry;
+    else if (col == kMaxBuckets) out[sl].dropped = carry;
+    else out[sl].above = carry;
   }
   if (threadIdx.x == 0) {
-    for (int b = 0; b < kMaxBuckets; ++b) out[sl].count[b] = tot[b];
-    out[sl].erase_max = erase_max;
-    out[sl].vmax2 = vmax2;
+    out[sl].erase_max = erase_index(rho2, in[sl], vmax2_bits[sl]);
+    out[sl].vmax2 = fmaxf(in[sl].prev_vmax2, __uint_as_float(vmax2_bits[sl]));
   }
 }
 
@@ -167,7 +203,8 @@ template <bool kBf16>
 __global__ void __launch_bounds__(256)
 bucket_scatter_kernel(Geom G, Arena A, const void* __restrict__ Ksrc, const void* __restrict__ Vsrc, int n, int chunks,
                       int n_buckets, const int8_t* __restrict__ slot, const int32_t* __restrict__ rank,
-                      const float* __restrict__ ns, const BucketDst* __restrict__ dst) {
+                      const int32_t* __restrict__ chunk_base, int n_chunks, const float* __restrict__ ns,
+                      const BucketDst* __restrict__ dst) {
   const int sl = blockIdx.y;
   const int rows_per_pass = blockDim.x / chunks;
   const int row_in = threadIdx.x / chunks, piece = threadIdx.x % chunks;
@@ -184,7 +221,7 @@ bucket_scatter_kernel(Geom G, Arena A, const void* __restrict__ Ksrc, const void
     int rk = 0;
     if (b >= 0) {
       const BucketDst D = dst[sl * n_buckets + b];
-      rk = rank[(size_t)sl * n + r];
+      rk = rank[(size_t)sl * n + r] + chunk_base[((size_t)sl * n_chunks + r / kScanChunk) * kCountCols + b];
       row = D.dst_row + rk;
       const uint4 kk = sK[(size_t)r * chunks + piece];
       const uint4 vv = sV[(size_t)r * chunks + piece];
@@ -204,26 +241,35 @@ bucket_scatter_kernel(Geom G, Arena A, const void* __restrict__ Ksrc, const void
 
 }  // namespace
 
+int bucket_scan_chunks(int n) { return (n + kScanChunk - 1) / kScanChunk; }
+size_t bucket_chunk_count_ints(int n_sl, int n) { return (size_t)n_sl * bucket_scan_chunks(n) * kCountCols; }
+
 cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, int n_buckets, int i_top, float rho2,
                                 const BucketIn* in, unsigned* vmax2_bits, float* ns, int8_t* slot, int32_t* rank,
-                                BucketOut* out, cudaStream_t st) {
+                                int32_t* chunk_cnt, BucketOut* out, cudaStream_t st) {
   const int chunks = G.d * (G.is_bf16 ? 2 : 4) / 16;
   cudaError_t e = cudaMemsetAsync(vmax2_bits, 0, sizeof(unsigned) * n_sl, st);
   if (e != cudaSuccess) return e;
   dim3 grid((n + kRowsPerBlock - 1) / kRowsPerBlock, n_sl);
   if (G.is_bf16) bucket_norms_kernel<true><<<grid, 256, 0, st>>>(V, n, chunks, ns, vmax2_bits);
   else bucket_norms_kernel<false><<<grid, 256, 0, st>>>(V, n, chunks, ns, vmax2_bits);
-  bucket_scan_kernel<<<n_sl, kScanThreads, 0, st>>>(ns, n, n_buckets, i_top, rho2, in, vmax2_bits, slot, rank, out);
+  const int n_chunks = bucket_scan_chunks(n);
+  bucket_scan_kernel<<<dim3(n_chunks, n_sl), kScanThreads, 0, st>>>(ns, n, n_chunks, n_buckets, i_top, rho2, in, vmax2_bits,
+                                                                   slot, rank, chunk_cnt);
+  bucket_prefix_kernel<<<n_sl, kCountCols * 32, 0, st>>>(n_chunks, rho2, in, vmax2_bits, chunk_cnt, out);
   return cudaGetLastError();
 }
 
 cudaError_t launch_bucket_scatter(const Geom& G, const Arena& A, const void* K, const void* V, int n_sl, int n,
-                                  int n_buckets, const int8_t* slot, const int32_t* rank, const float* ns,
-                                  const BucketDst* dst, cudaStream_t st) {
+                                  int n_buckets, const int8_t* slot, const int32_t* rank, const int32_t* chunk_base,
+                                  const float* ns, const BucketDst* dst, cudaStream_t st) {
   const int chunks = G.d * (G.is_bf16 ? 2 : 4) / 16;
+  const int n_chunks = bucket_scan_chunks(n);
   dim3 grid((n + kRowsPerBlock - 1) / kRowsPerBlock, n_sl);
-  if (G.is_bf16) bucket_scatter_kernel<true><<<grid, 256, 0, st>>>(G, A, K, V, n, chunks, n_buckets, slot, rank, ns, dst);
-  else bucket_scatter_kernel<false><<<grid, 256, 0, st>>>(G, A, K, V, n, chunks, n_buckets, slot, rank, ns, dst);
+  if (G.is_bf16)
+    bucket_scatter_kernel<true><<<grid, 256, 0, st>>>(G, A, K, V, n, chunks, n_buckets, slot, rank, chunk_base, n_chunks, ns, dst);
+  else
+    bucket_scatter_kernel<false><<<grid, 256, 0, st>>>(G, A, K, V, n, chunks, n_buckets, slot, rank, chunk_base, n_chunks, ns, dst);
   return cudaGetLastError();
 }
 

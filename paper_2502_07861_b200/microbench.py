@@ -2,6 +2,7 @@
 
     python -m paper_2502_07861_b200.microbench decode   --batch 32 --cache-len 8192 --levels 2 [--two-instance]
     python -m paper_2502_07861_b200.microbench compress --streams 8 --context 32768 --block 1024 --levels 2
+    python -m paper_2502_07861_b200.microbench bucket   --streams 8 --context 32768 --buckets 5
 
 Prints one JSON line per run.  Inputs are drawn on the device (torch.randn), which is enough
 for timing; parity is the tests' job.
@@ -116,6 +117,59 @@ def run_compress(a):
     ctx.close()
 
 
+def run_bucket(a):
+    """Algorithm 1's bucketing step (value norms, stable partition, scatter into the per-bucket slots),
+    then compress of all slots and the merged decode over them."""
+    S, d, n, t, T, nb = a.streams, a.head_dim, a.context, a.block, a.levels, a.buckets
+    ctx = bk.Context(n_seqs=1, n_layers=nb + 1, n_kv_heads=S, n_q_heads=S * 4, head_dim=d, dtype="bf16", block=t,
+                     levels=T, max_tokens=n)
+    K = torch.randn(1, S, n, d, device="cuda", dtype=torch.float32)
+    K[..., :4] *= 10.0
+    K = K.to(torch.bfloat16)
+    scale = torch.exp2(-float(nb) * torch.rand(1, S, n, 1, device="cuda"))     # norms spread over the nb octaves
+    V = (torch.randn(1, S, n, d, device="cuda", dtype=torch.float32) * scale).to(torch.bfloat16)
+    i_top = 4                                                                    # ||v|| <= 16
+    q = torch.randn(1, S * 4, d, device="cuda").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    t_route = t_comp = t_dec = 0.0
+    ctx.profile_enable(True)
+    for i in range(a.iters + 2):
+        ctx.reset()
+        flush.fill_(i & 255)
+        if i == 2:
+            ctx.profile_read()
+        ev[0].record()
+        counts = ctx.stream_append_layer_bucketed(0, nb, i_top, K, V)
+        ev[1].record()
+        ctx.stream_append_layer_keys(nb, K)
+        ctx.compress()
+        ev[2].record()
+        ctx.decode_attn_merged(list(range(nb)), [nb], q, out)
+        ev[3].record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            t_route += ev[0].elapsed_time(ev[1]); t_comp += ev[1].elapsed_time(ev[2]); t_dec += ev[2].elapsed_time(ev[3])
+    prof = ctx.profile_read()
+    hbm, _, src = _peaks()
+    kept = int(counts[:, :nb].sum())
+    # read V for the norms, read K and V of the kept rows, write them: 2 bytes per element
+    route_bytes = S * n * d * 2 + kept * 4 * d * 2
+    # class 0 also holds the keys-only append of the denominator slot: one launch per iteration, subtracted by count
+    st = ctx.stats()
+    print(json.dumps(dict(kernel="bucket_route", streams=S, context=n, buckets=nb, block=t, levels=T,
+                          rows_kept=kept, rows_dropped=int(counts[:, nb].sum()), per_slot=counts[:, :nb].sum(0).tolist(),
+                          route_call_ms=t_route / a.iters, algorithmic_bytes=route_bytes,
+                          achieved_gbs=route_bytes / (t_route / a.iters * 1e-3) / 1e9, peak_gbs=hbm,
+                          frac=route_bytes / (t_route / a.iters * 1e-3) / 1e9 / hbm,
+                          append_class_launches=prof["append"][0] // a.iters, append_class_ms=prof["append"][1] / a.iters,
+                          compress_ms=t_comp / a.iters, merged_decode_ms=t_dec / a.iters,
+                          token_heads_per_s=S * n / ((t_route + t_comp) / a.iters * 1e-3),
+                          device_status=st["device_status"], peak_source=src)))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -140,10 +194,18 @@ def main():
     c.add_argument("--gram-path", type=int, default=0)
     c.add_argument("--c-override", type=float, default=0.0)
     c.add_argument("--outliers", type=int, default=1)
+    b = sub.add_parser("bucket")
+    b.add_argument("--streams", type=int, default=8)
+    b.add_argument("--head-dim", type=int, default=128)
+    b.add_argument("--context", type=int, default=32768)
+    b.add_argument("--block", type=int, default=1024)
+    b.add_argument("--levels", type=int, default=2)
+    b.add_argument("--buckets", type=int, default=5)
+    b.add_argument("--iters", type=int, default=10)
     a = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("microbench needs a CUDA device")
-    (run_decode if a.cmd == "decode" else run_compress)(a)
+    {"decode": run_decode, "compress": run_compress, "bucket": run_bucket}[a.cmd](a)
 
 
 if __name__ == "__main__":
