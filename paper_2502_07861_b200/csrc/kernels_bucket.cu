@@ -70,8 +70,17 @@ bucket_norms_kernel(const void* __restrict__ V, int n, int chunks, float* __rest
     mx = fmaxf(mx, s);
   }
   mx = warp_max(mx);
-  // squared norms are >= 0, so their bit patterns order like the values
-  if ((threadIdx.x & 31) == 0 && mx > 0.f) atomicMax(vmax2_bits + sl, __float_as_uint(mx));
+  __shared__ float warp_mx[8];
+  if ((threadIdx.x & 31) == 0) warp_mx[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, warp_mx[w]);
+    // squared norms are >= 0, so their bit patterns order like the values; one atomic per CTA,
+    // and none once the stream's maximum is already at least this large
+    const unsigned bits = __float_as_uint(mx);
+    if (bits > *reinterpret_cast<volatile unsigned*>(vmax2_bits + sl)) atomicMax(vmax2_bits + sl, bits);
+  }
 }
 
 // The bucket index of a squared norm: the smallest i with 4^i >= ns (ns > 0).
