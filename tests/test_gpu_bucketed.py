@@ -154,3 +154,70 @@ def test_bucketed_per_stream_entry_and_refusals(cuda_lib):
         assert sum(ctx.level_sizes(0, s, 0)) == 0                 # the other head's instances are untouched
     with pytest.raises(Exception):
         ctx.stream_append_bucketed(0, 2, 4, 4, 1, Kd, Vd)         # slots beyond the context's layers
+
+
+def test_bucketed_llama_layer_full_size_sampled_instances(cuda_lib):
+    """The one-layer Llama-3.1-8B-shaped workload (8 KV heads x 32768 tokens, d = 128, bf16, block
+    1024, T = 2) through the bucketed path: routing of every row of every stream against a direct
+    evaluation of the bucket rule, size-independent properties of every instance, teacher-forced
+    replay of two sampled instances, and the merged decode of a sampled head."""
+    B, H, g, d, n, t, T, nb, i_top = 1, 8, 4, 128, 32768, 1024, 2, 4, 4
+    K = np.empty((B, H, n, d), np.float32)
+    V = np.empty_like(K)
+    for h in range(H):
+        k, v = synth.stream_kv("llama", 1002, 0, 0, h, n, d, "bf16")
+        scale = 2.0 ** np.random.default_rng([1002, h]).uniform(-3.9, 0.0, n)
+        K[0, h], V[0, h] = k, synth.round_to((v * scale[:, None]).astype(np.float32), "bf16")
+    # rows whose norm sits within rounding of a bucket boundary are moved off it (see _not_borderline)
+    frac = 0.5 * np.log2(np.sum(V.astype(np.float64) ** 2, -1))
+    near = np.abs(frac - np.round(frac)) <= 1e-4
+    V[near] = synth.round_to(V[near] * np.float32(1.0625), "bf16")
+    _not_borderline(V, 0.0)
+    ns = np.sum(V.astype(np.float64) ** 2, -1)
+    want = i_top - np.ceil(0.5 * np.log2(ns)).astype(np.int64)           # the bucket rule, written out
+    assert want.min() >= 0
+    want = np.where(want < nb, want, -1)
+    ctx = cuda_lib.Context(n_seqs=B, n_layers=nb + 1, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=t,
+                           levels=T, max_tokens=n, seed=7)
+    ctx.debug_enable(True)
+    Kd, Vd = to_device(K, "bf16"), to_device(V, "bf16")
+    counts, slots = ctx.stream_append_layer_bucketed(0, nb, i_top, Kd, Vd, want_slots=True)
+    ctx.stream_append_layer_keys(nb, Kd)
+    ctx.compress()
+    assert np.array_equal(slots.cpu().numpy(), want)
+    for h in range(H):
+        assert [int(x) for x in counts[h]] == [int(np.sum(want[0, h] == s)) for s in range(nb)] + [int(np.sum(want[0, h] < 0))]
+        for s in range(nb):
+            m = int(counts[h, s])
+            _, _, w, idx = ctx.cache_view(0, s, h)
+            sizes = ctx.level_sizes(0, s, h)
+            assert float(w.sum()) == m                                   # Theorem 3.3's weights stand for every row
+            assert sizes[0] == m % t
+            assert sizes[T] == (m // (2 * t)) * (t // 2) and torch.all(idx[: sizes[T]][1:] > idx[: sizes[T]][:-1])
+    st = ctx.stats()
+    assert st["device_status"] == 0
+    from oracle import OracleStream
+    from parity_util import check_stream, gpu_call_records, oracle_params
+    tot = marg = 0
+    for (h, s) in ((2, 1), (5, 3)):
+        rows = np.flatnonzero(want[0, h] == s)
+        rec = gpu_call_records(ctx, 0, s, h, len(rows) // t)
+        o = OracleStream(oracle_params(ctx, 0, s, h))
+        for (lvl, od), (eta, _, _) in rec.items():
+            o.force_eta(lvl, od, eta)
+        o.append(K[0, h][rows], V[0, h][rows])
+        o.compress()
+        a, b = check_stream(ctx, 0, s, h, o, rec, 2e-4)
+        tot, marg = tot + a, marg + b
+    assert tot > 0 and marg <= 1e-3 * tot
+    # merged decode of every head against the oracle's ratio evaluated on the library's own sets
+    q = synth.queries(1002, 0, 0, B, H * g, d, "bf16")
+    out = ctx.decode_attn_merged(list(range(nb)), [nb], to_device(q, "bf16")).float().cpu().numpy()
+    for h in (0, 5):
+        views = []
+        for s in range(nb + 1):
+            Kg, Vg, wg, _ = ctx.cache_view(0, s, h)
+            views.append((Kg.float().cpu().numpy().astype(np.float64), Vg.float().cpu().numpy().astype(np.float64),
+                          wg.cpu().numpy().astype(np.float64)))
+        ref = oracle.merged_estimate(views[:nb], [views[nb]], q[0, h * g:(h + 1) * g])
+        assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3
