@@ -635,6 +635,9 @@ static int pick_splits(balancekv_ctx* c, int layer) {
   const int tile_tokens = 16384 / (f.head_dim * c->esz);
   const int64_t tiles = (max_rows + tile_tokens - 1) / tile_tokens + f.levels;
   int splits = (int)std::max<int64_t>(1, std::min<int64_t>(c->max_splits, (tiles + 1) / 2));
+  // the fewest splits with the same number of tiles per CTA: the tile phase is as long, the combine shorter
+  const int64_t tiles_per = std::max<int64_t>(1, (tiles + splits - 1) / splits);
+  splits = (int)std::max<int64_t>(1, (tiles + tiles_per - 1) / tiles_per);
   if (f.decode_splits > 0) splits = std::min(f.decode_splits, c->max_splits);
   return splits;
 }
