@@ -99,7 +99,9 @@ struct balancekv_ctx {
   // stream_step_host: q | k_new | v_new of a step packed into one pinned slot, one copy to the device
   static constexpr int kStepSlots = 64;
   char* step_host = nullptr;            // pinned, kStepSlots slots
-  char* step_dev_in = nullptr;          // q | k | v
+  char* step_dev_in = nullptr;          // q | k | v, kStepSlots slots as well
+  cudaStream_t step_copy_stream = nullptr;   // the transfers run beside the caller's stream
+  cudaEvent_t step_used_ev[kStepSlots] = {}; // the step's kernel has finished (its slots may be reused)
   void* step_dev_out = nullptr;
   size_t step_slot_bytes = 0;
   cudaEvent_t step_ev[kStepSlots] = {};
@@ -370,6 +372,9 @@ int balancekv_destroy(balancekv_ctx* c) {
   if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
   if (c->h_ring) cudaFreeHost(c->h_ring);
   if (c->step_host) cudaFreeHost(c->step_host);
+  if (c->step_copy_stream) cudaStreamDestroy(c->step_copy_stream);
+  for (cudaEvent_t e : c->step_used_ev)
+    if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->step_ev)
     if (e) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i)
@@ -799,22 +804,28 @@ int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, 
     c->step_slot_bytes = (qb + 2 * kb + 255) / 256 * 256;
     BKV_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->step_host), c->step_slot_bytes * balancekv_ctx::kStepSlots,
                            cudaHostAllocDefault));
-    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->step_dev_in), c->step_slot_bytes));
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->step_dev_in), c->step_slot_bytes * balancekv_ctx::kStepSlots));
     BKV_CUDA(cudaMalloc(&c->step_dev_out, qb));
-    c->bytes_resident += c->step_slot_bytes + qb;
+    c->bytes_resident += c->step_slot_bytes * balancekv_ctx::kStepSlots + qb;
     for (cudaEvent_t& e : c->step_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    for (cudaEvent_t& e : c->step_used_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    BKV_CUDA(cudaStreamCreateWithFlags(&c->step_copy_stream, cudaStreamNonBlocking));
   }
-  // The three small inputs travel as one copy: packed into a pinned slot on the host (a slot is
-  // reused only after the copy that read it has finished), then one host-to-device transfer.
+  // The three small inputs travel as one copy: packed into a pinned slot on the host, then one
+  // host-to-device transfer into the slot's device twin on the library's copy stream, so that the
+  // transfer of a step runs while the previous step's kernel does; the kernel waits for its
+  // transfer through an event.  A slot pair is reused only after the kernel that read it has finished.
   const int slot = (int)(c->step_count % balancekv_ctx::kStepSlots);
-  if (c->step_count >= (unsigned long long)balancekv_ctx::kStepSlots) BKV_CUDA(cudaEventSynchronize(c->step_ev[slot]));
+  if (c->step_count >= (unsigned long long)balancekv_ctx::kStepSlots) BKV_CUDA(cudaEventSynchronize(c->step_used_ev[slot]));
   ++c->step_count;
   char* h = c->step_host + (size_t)slot * c->step_slot_bytes;
+  char* dev_in = c->step_dev_in + (size_t)slot * c->step_slot_bytes;
   std::memcpy(h, q_host, qb);
   std::memcpy(h + qb, k_host, kb);
   std::memcpy(h + qb + kb, v_host, kb);
-  BKV_CUDA(cudaMemcpyAsync(c->step_dev_in, h, qb + 2 * kb, cudaMemcpyHostToDevice, st));
-  BKV_CUDA(cudaEventRecord(c->step_ev[slot], st));
+  BKV_CUDA(cudaMemcpyAsync(dev_in, h, qb + 2 * kb, cudaMemcpyHostToDevice, c->step_copy_stream));
+  BKV_CUDA(cudaEventRecord(c->step_ev[slot], c->step_copy_stream));
+  BKV_CUDA(cudaStreamWaitEvent(st, c->step_ev[slot], 0));
   // A pinned (mapped) result buffer is written by the kernel itself: the 8 KB of a step then need
   // no transfer of their own.  Pageable memory goes through the device buffer and a copy.
   void* out_dev = nullptr;
@@ -826,8 +837,8 @@ int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, 
     else
       (void)cudaGetLastError();
   }
-  int rc = balancekv_stream_step(c, layer, c->step_dev_in, c->step_dev_in + qb, c->step_dev_in + qb + kb,
-                                 out_dev ? out_dev : c->step_dev_out, stream);
+  int rc = balancekv_stream_step(c, layer, dev_in, dev_in + qb, dev_in + qb + kb, out_dev ? out_dev : c->step_dev_out, stream);
+  BKV_CUDA(cudaEventRecord(c->step_used_ev[slot], st));
   if (rc) return rc;
   if (!out_dev) BKV_CUDA(cudaMemcpyAsync(out_host, c->step_dev_out, qb, cudaMemcpyDeviceToHost, st));
   return BALANCEKV_OK;
