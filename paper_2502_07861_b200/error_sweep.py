@@ -4,6 +4,7 @@ single-layer ablations (relative error ||z - Attn|| / ||Attn|| over T and t), on
 keys and values instead of the paper's prompts.
 
     python -m paper_2502_07861_b200.error_sweep --recipe clustered --n 8192 --blocks 64,256 --levels 1,2,3 --seeds 5
+    python -m paper_2502_07861_b200.error_sweep --recipe clustered_norms --buckets 4 --n 16384 --blocks 64,256 --levels 1,2 --seeds 5
 
 Everything runs through the library: BalanceKV = append + compress + decode; uniform sampling = a
 cache loaded directly at level T with a random subset and weights 2^T; exact = a context with T = 0.
@@ -22,7 +23,7 @@ from . import binding as bk
 def make_kv(recipe, seed, H, n, d):
     """bf16 K, V [1, H, n, d] on the device."""
     g = torch.Generator(device="cuda").manual_seed(seed)
-    if recipe == "clustered":
+    if recipe in ("clustered", "clustered_norms"):
         # near-duplicate keys on a few equal-norm centres, values tied to the cluster: the case in
         # which a balanced half beats a random half
         unit = lambda a: a / a.norm(dim=-1, keepdim=True)
@@ -31,6 +32,9 @@ def make_kv(recipe, seed, H, n, d):
         lab = torch.randint(0, 8, (H, n), device="cuda", generator=g)
         K = torch.gather(centres, 1, lab[..., None].expand(H, n, d)) + 0.02 * torch.randn(H, n, d, device="cuda", generator=g)
         V = torch.gather(vals, 1, lab[..., None].expand(H, n, d)) + 0.02 * torch.randn(H, n, d, device="cuda", generator=g)
+        if recipe == "clustered_norms":
+            # value norms spread over three octaves: the case Algorithm 1's buckets are made for
+            V = V * torch.exp2(-3.0 * torch.rand(H, n, 1, device="cuda", generator=g))
         Q = 0.5 * (centres[:, :4] + centres[:, 4:])                       # [H, 4, d] queries between two clusters
     else:
         mu = 0.5 * torch.randn(H, 1, d, device="cuda", generator=g)
@@ -49,7 +53,7 @@ def rel_err(z, ref):
     return float(((z - ref).norm(dim=-1) / ref.norm(dim=-1).clamp_min(1e-30)).mean())
 
 
-def run_point(recipe, seed, H, n, d, t, T, c_small, center):
+def run_point(recipe, seed, H, n, d, t, T, c_small, center, buckets=0):
     K, V, q = make_kv(recipe, seed, H, n, d)
     common = dict(n_seqs=1, n_layers=1, n_kv_heads=H, n_q_heads=4 * H, head_dim=d, dtype="bf16", max_tokens=n)
     exact_ctx = bk.Context(block=t, levels=0, **common)
@@ -67,6 +71,21 @@ def run_point(recipe, seed, H, n, d, t, T, c_small, center):
         assert st["device_status"] == 0
         out[name + "_fails"] = st["walk_fails"]
         ctx.close()
+    if buckets > 0:
+        # Algorithm 1 in full: one MergeAndReduce instance per value-norm bucket for the numerator
+        # (||v|| <= 2 assumed by the recipes: i_top = 1), a keys-only instance for the denominator
+        full = dict(common, n_layers=buckets + 1)
+        for name, c in (("algorithm1_paper_c", 0.0), ("algorithm1_small_c", c_small)):
+            ctx = bk.Context(block=t, levels=T, seed=seed, c_override=c, center_keys=center, **full)
+            counts = ctx.stream_append_layer_bucketed(0, buckets, 1, K, V)
+            ctx.stream_append_layer_keys(buckets, K)
+            ctx.compress()
+            out[name] = rel_err(ctx.decode_attn_merged(list(range(buckets)), [buckets], q), exact)
+            st = ctx.stats()
+            assert st["device_status"] == 0
+            out[name + "_stored"] = st["tokens_stored"] / (H * (buckets + 1))   # rows per stream over all instances
+            out[name + "_dropped"] = int(counts[:, buckets].sum())
+            ctx.close()
     g = torch.Generator(device="cuda").manual_seed(10_000 + seed)
     keep = n >> T
     idx = torch.stack([torch.randperm(n, device="cuda", generator=g)[:keep].sort().values for _ in range(H)])   # [H, keep]
@@ -81,7 +100,7 @@ def run_point(recipe, seed, H, n, d, t, T, c_small, center):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--recipe", default="clustered", choices=("clustered", "llama"))
+    ap.add_argument("--recipe", default="clustered", choices=("clustered", "clustered_norms", "llama"))
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--heads", type=int, default=4)
     ap.add_argument("--head-dim", type=int, default=128)
@@ -90,6 +109,7 @@ def main():
     ap.add_argument("--seeds", type=int, default=10)
     ap.add_argument("--small-c", type=float, default=0.25)
     ap.add_argument("--center-keys", type=int, default=0)
+    ap.add_argument("--buckets", type=int, default=0, help="> 0: also Algorithm 1 with this many value-norm buckets")
     a = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("error_sweep needs a CUDA device")
@@ -99,7 +119,7 @@ def main():
                 continue
             acc = {}
             for seed in range(a.seeds):
-                for k, v in run_point(a.recipe, seed, a.heads, a.n, a.head_dim, t, T, a.small_c, a.center_keys).items():
+                for k, v in run_point(a.recipe, seed, a.heads, a.n, a.head_dim, t, T, a.small_c, a.center_keys, a.buckets).items():
                     acc[k] = acc.get(k, 0.0) + v / a.seeds
             print(json.dumps(dict(recipe=a.recipe, n=a.n, block=t, levels=T, rate=2.0 ** -T, seeds=a.seeds,
                                   center_keys=a.center_keys, small_c=a.small_c, **{k: round(v, 6) for k, v in acc.items()})))
