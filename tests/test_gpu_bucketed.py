@@ -221,3 +221,18 @@ def test_bucketed_llama_layer_full_size_sampled_instances(cuda_lib):
                           wg.cpu().numpy().astype(np.float64)))
         ref = oracle.merged_estimate(views[:nb], [views[nb]], q[0, h * g:(h + 1) * g])
         assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3
+
+
+def test_error_sweep_point_buckets_beat_uniform_on_mixed_value_norms(cuda_lib):
+    """One point of the error-against-rate sweep with value norms spread over three octaves: a walk
+    that is not a fair coin needs Algorithm 1's buckets (without them it is no better than uniform
+    sampling, with them clearly better)."""
+    from paper_2502_07861_b200 import error_sweep
+
+    acc = {}
+    for seed in range(4):
+        for k, v in error_sweep.run_point("clustered_norms", seed, 2, 8192, 128, 128, 1, 0.25, 0, buckets=4).items():
+            acc[k] = acc.get(k, 0.0) + v / 4
+    assert acc["algorithm1_small_c"] < 0.8 * acc["uniform"]
+    assert acc["algorithm1_small_c"] < 0.8 * acc["balancekv_small_c"]
+    assert 0.5 * acc["uniform"] < acc["algorithm1_paper_c"] < 2.0 * acc["uniform"]
