@@ -513,16 +513,49 @@ int balancekv_cache_load_level(balancekv_ctx* c, int layer, int level, const voi
 // level-0 remainder moves and the segment-table update.
 static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
   const Geom& G = c->G;
+  // Every descriptor array of the batch (the calls of each level, the remainder moves, the segment
+  // updates) travels in one transfer ahead of the first kernel, so that no copy sits between two
+  // kernels of the batch; if they do not fit one half of the ring they go array by array.
+  auto pad = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  size_t total = 0;
+  for (int l = 0; l < G.T; ++l) {
+    if (c->debug)
+      for (CallDesc& d : P.levels[l]) d.dbg_off = dbg_offset(c, d.stream, l, d.ordinal);
+    total += pad(P.levels[l].size() * sizeof(CallDesc));
+  }
+  const size_t off_moves = total;
+  total += pad(P.moves.size() * sizeof(MoveDesc));
+  const size_t off_segs = total;
+  total += pad(P.segs.size() * sizeof(SegUpdate));
+  char* d_all = nullptr;
+  if (total > 0 && total <= c->ring_half) {
+    std::vector<char> host(total);
+    size_t off = 0;
+    for (int l = 0; l < G.T; ++l) {
+      const size_t b = P.levels[l].size() * sizeof(CallDesc);
+      if (b) std::memcpy(host.data() + off, P.levels[l].data(), b);
+      off += pad(b);
+    }
+    if (!P.moves.empty()) std::memcpy(host.data() + off_moves, P.moves.data(), P.moves.size() * sizeof(MoveDesc));
+    if (!P.segs.empty()) std::memcpy(host.data() + off_segs, P.segs.data(), P.segs.size() * sizeof(SegUpdate));
+    void* dv = nullptr;
+    int rc = ring_push(c, host.data(), total, st, &dv);
+    if (rc) return rc;
+    d_all = static_cast<char*>(dv);
+  }
+  size_t off_level = 0;
   for (int l = 0; l < G.T; ++l) {
     std::vector<CallDesc>& calls = P.levels[l];
+    const size_t level_base = off_level;
+    off_level += pad(calls.size() * sizeof(CallDesc));
     if (calls.empty()) continue;
-    if (c->debug)
-      for (CallDesc& d : calls) d.dbg_off = dbg_offset(c, d.stream, l, d.ordinal);
     for (size_t first = 0; first < calls.size(); first += c->max_calls) {
       const int n = (int)std::min<size_t>(c->max_calls, calls.size() - first);
-      void* d_calls = nullptr;
-      int rc = ring_push(c, calls.data() + first, (size_t)n * sizeof(CallDesc), st, &d_calls);
-      if (rc) return rc;
+      void* d_calls = d_all ? d_all + level_base + first * sizeof(CallDesc) : nullptr;
+      if (!d_all) {
+        int rc = ring_push(c, calls.data() + first, (size_t)n * sizeof(CallDesc), st, &d_calls);
+        if (rc) return rc;
+      }
       const CallDesc* dc = static_cast<const CallDesc*>(d_calls);
       // the tensor-core walk kernel takes the radii from the stored row norms itself
       const bool need_radii = (G.center_keys || G.fixed_rk2 <= 0.f || G.fixed_rv2 <= 0.f) &&
@@ -550,17 +583,21 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
     }
   }
   if (!P.moves.empty()) {
-    void* d_moves = nullptr;
-    int rc = ring_push(c, P.moves.data(), P.moves.size() * sizeof(MoveDesc), st, &d_moves);
-    if (rc) return rc;
+    void* d_moves = d_all ? d_all + off_moves : nullptr;
+    if (!d_all) {
+      int rc = ring_push(c, P.moves.data(), P.moves.size() * sizeof(MoveDesc), st, &d_moves);
+      if (rc) return rc;
+    }
     ProfScope ps(c, 5, st);
     BKV_CUDA(launch_move(G, c->A, static_cast<const MoveDesc*>(d_moves), (int)P.moves.size(), P.max_move_rows, st));
     c->kernels_launched++;
   }
   if (!P.segs.empty()) {
-    void* d_segs = nullptr;
-    int rc = ring_push(c, P.segs.data(), P.segs.size() * sizeof(SegUpdate), st, &d_segs);
-    if (rc) return rc;
+    void* d_segs = d_all ? d_all + off_segs : nullptr;
+    if (!d_all) {
+      int rc = ring_push(c, P.segs.data(), P.segs.size() * sizeof(SegUpdate), st, &d_segs);
+      if (rc) return rc;
+    }
     ProfScope ps(c, 5, st);
     BKV_CUDA(launch_seg_update(c->A, static_cast<const SegUpdate*>(d_segs), (int)P.segs.size(), st));
     c->kernels_launched++;
