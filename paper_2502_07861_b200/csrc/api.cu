@@ -26,6 +26,10 @@ void decode_mma_release(void* maps);
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
                                     float* scratch, int splits, int* status, const void* maps, int keys_only,
                                     cudaStream_t st);
+cudaError_t launch_decode_parts_mma_slots(const Geom& G, const Arena& A, const int* slot_layers, int n_slots,
+                                          unsigned keys_mask, const void* q, float* raw_acc, float* raw_ml, float* scratch,
+                                          size_t z_stride_words, int splits, int* status, const void* maps,
+                                          cudaStream_t st);
 cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, unsigned num_mask, unsigned den_mask,
                                 void* out, int n_heads, int d, cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
@@ -109,6 +113,8 @@ struct balancekv_ctx {
   // two-instance estimator: un-normalised parts of the numerator and denominator instances, unit values
   float* two_acc = nullptr;             // [BALANCEKV_MAX_MERGE][B, Hq, d] value sums per merged slot
   float* two_ml = nullptr;              // [BALANCEKV_MAX_MERGE][B, Hq, 2] (max, sum) per merged slot
+  float* two_scratch = nullptr;         // [BALANCEKV_MAX_MERGE] split-K scratch blocks (tickets + partial rows)
+  size_t two_scratch_words = 0;         // 4-byte words per block
   void* unit_V = nullptr;               // rows (1, 0, ..., 0) for balancekv_stream_append_layer_keys
   size_t unit_rows = 0;
 
@@ -363,7 +369,7 @@ int balancekv_destroy(balancekv_ctx* c) {
   decode_mma_release(c->decode_maps);
   void* ptrs[] = {c->A.K, c->A.V, c->A.idx, c->A.seg, c->A.nrm, c->d_stats, c->d_tokshift, c->d_eta, c->d_fail, c->d_status,
                   c->d_decode_scratch, c->d_ring, c->dbg_eta, c->dbg_S, c->dbg_p, c->view_K, c->view_V, c->view_w,
-                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->unit_V};
+                  c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->two_scratch, c->unit_V};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out, c->bkt_chunk_cnt};
@@ -774,16 +780,30 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_acc), sizeof(float) * (size_t)n_heads * d * BALANCEKV_MAX_MERGE));
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_ml), sizeof(float) * (size_t)n_heads * 2 * BALANCEKV_MAX_MERGE));
     c->bytes_resident += sizeof(float) * (size_t)n_heads * (d + 2) * BALANCEKV_MAX_MERGE;
+    // one split-K scratch block per slot, so that all slots go in one launch; tickets start at zero
+    const size_t block_bytes = (decode_scratch_bytes(c->G, c->max_splits) + 255) & ~(size_t)255;
+    BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_scratch), block_bytes * BALANCEKV_MAX_MERGE));
+    BKV_CUDA(cudaMemsetAsync(c->two_scratch, 0, block_bytes * BALANCEKV_MAX_MERGE, st));
+    c->two_scratch_words = block_bytes / 4;
+    c->bytes_resident += block_bytes * BALANCEKV_MAX_MERGE;
   }
+  // One launch over all slots (grid z = slot).  The split factor is the largest any slot asks for,
+  // bounded so that the whole grid stays within one wave of two CTAs per SM where it can.
+  int splits = 1;
+  unsigned keys_mask = 0;
   for (int p = 0; p < n_parts; ++p) {
+    splits = std::max(splits, pick_splits(c, slots[p]));
+    if (!((num_mask >> p) & 1u)) keys_mask |= 1u << p;     // a slot that only enters the denominator: values are not read
+  }
+  const int n_sl = c->cfg.n_seqs * c->cfg.n_kv_heads;
+  splits = std::max(1, std::min(splits, 2 * c->sm_count / std::max(1, n_sl * n_parts)));
+  {
     ProfScope ps(c, 4, st);
-    const int keys_only = ((num_mask >> p) & 1u) ? 0 : 1;  // a slot that only enters the denominator: values are not read
-    BKV_CUDA(launch_decode_parts_mma(c->G, c->A, slots[p], q, c->two_acc + (size_t)p * n_heads * d,
-                                     c->two_ml + (size_t)p * n_heads * 2, c->d_decode_scratch, pick_splits(c, slots[p]),
-                                     c->d_status, c->decode_maps, keys_only, st));
+    BKV_CUDA(launch_decode_parts_mma_slots(c->G, c->A, slots, n_parts, keys_mask, q, c->two_acc, c->two_ml, c->two_scratch,
+                                           c->two_scratch_words, splits, c->d_status, c->decode_maps, st));
   }
   BKV_CUDA(launch_merged_ratio(c->two_acc, c->two_ml, n_parts, num_mask, den_mask, out, n_heads, d, st));
-  c->kernels_launched += n_parts + 1;
+  c->kernels_launched += 2;
   return BALANCEKV_OK;
 }
 

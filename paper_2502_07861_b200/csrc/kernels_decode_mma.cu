@@ -113,6 +113,14 @@ struct StepAppend {
   // dependent global read at the start of a latency-bound launch.  n_seg = 0: read the table.
   int n_seg;
   Seg seg[kMaxLevels + 1];
+  // One launch over several layer slots (decode merged over slots): blockIdx.z selects the slot.
+  // n_slots = 0: a launch over the one slot `layer`.  z_stride: 4-byte words between the scratch
+  // blocks (tickets, partial rows) of consecutive slots; raw_acc / raw_ml advance by one
+  // [B, H g, d] / [B, H g, 2] block per slot; bit z of keys_mask = keys_only of slot z.
+  int n_slots;
+  int slot_layer[8];
+  unsigned keys_mask;
+  unsigned z_stride;
 };
 
 struct TileRef {
@@ -137,8 +145,22 @@ __device__ inline TileRef locate_tile(int tile, const int* lvl_tiles, const Seg*
 
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
-                  float* __restrict__ part, unsigned* __restrict__ tickets, int* __restrict__ status, StepAppend ap,
-                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
+                  float* __restrict__ part_base, unsigned* __restrict__ tickets_base, int* __restrict__ status,
+                  const StepAppend ap, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
+  float* part = part_base;
+  unsigned* tickets = tickets_base;
+  float* raw_acc = ap.raw_acc;
+  float* raw_ml = ap.raw_ml;
+  int keys_only = ap.keys_only;
+  if (ap.n_slots) {
+    const int z = blockIdx.z;
+    layer = ap.slot_layer[z];
+    keys_only = (int)((ap.keys_mask >> z) & 1u);
+    part += (size_t)z * ap.z_stride;
+    tickets += (size_t)z * ap.z_stride;
+    raw_acc += (size_t)z * G.B * G.H * G.g * kD;
+    raw_ml += (size_t)z * G.B * G.H * G.g * 2;
+  }
   extern __shared__ unsigned char smem_raw[];
   unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(tiles + kStages * kStageBytes);
@@ -183,10 +205,10 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
     unsigned char* st = tiles + (size_t)(i % kStages) * kStageBytes;
     uint64_t* bar = &full[i % kStages];
-    mbar_expect_tx(bar, ap.keys_only ? kTensorBytes : kStageBytes);
+    mbar_expect_tx(bar, keys_only ? kTensorBytes : kStageBytes);
     tma_load_2d(st, &tmK, 0, (int)tr.row, bar);
     tma_load_2d(st + kHalf, &tmK, 64, (int)tr.row, bar);
-    if (!ap.keys_only) {
+    if (!keys_only) {
       tma_load_2d(st + kTensorBytes, &tmV, 0, (int)tr.row, bar);
       tma_load_2d(st + kTensorBytes + kHalf, &tmV, 64, (int)tr.row, bar);
     }
@@ -263,7 +285,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       const uint32_t pl[4] = {pack_bf16(x0 - bf16_lo(ph[0]), x1 - bf16_hi(ph[0])), 0u,
                               pack_bf16(x2 - bf16_lo(ph[2]), x3 - bf16_hi(ph[2])), 0u};
       // ---- O[16 x 128] += P[16 x 16] V[16 x 128]
-      if (!ap.keys_only)
+      if (!keys_only)
 #pragma unroll
       for (int nb = 0; nb < 8; ++nb) {
         uint32_t vb[4];
@@ -493,10 +515,10 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       acc.x = fmaf(__bfloat162float(v01.x), fN, acc.x); acc.y = fmaf(__bfloat162float(v01.y), fN, acc.y);
       acc.z = fmaf(__bfloat162float(v23.x), fN, acc.z); acc.w = fmaf(__bfloat162float(v23.y), fN, acc.w);
     }
-    if (ap.raw_acc) {
+    if (raw_acc) {
       const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
-      *reinterpret_cast<float4*>(ap.raw_acc + qh * kD + c) = acc;
-      if (c == 0) { ap.raw_ml[2 * qh] = cM[h]; ap.raw_ml[2 * qh + 1] = cL[h]; }
+      *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = acc;
+      if (c == 0) { raw_ml[2 * qh] = cM[h]; raw_ml[2 * qh + 1] = cL[h]; }
       continue;
     }
     const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
@@ -564,9 +586,28 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}};
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
                                                         tickets, status, ap, tm->k, tm->v);
+  return cudaGetLastError();
+}
+
+// The same for n_slots layer slots in one launch (grid z = slot): raw_acc / raw_ml hold one block per
+// slot, scratch one block of z_stride_words 4-byte words per slot (laid out as for a single slot).
+cudaError_t launch_decode_parts_mma_slots(const Geom& G, const Arena& A, const int* slot_layers, int n_slots,
+                                          unsigned keys_mask, const void* q, float* raw_acc, float* raw_ml, float* scratch,
+                                          size_t z_stride_words, int splits, int* status, const void* maps,
+                                          cudaStream_t st) {
+  if (!maps || !raw_acc || !raw_ml || n_slots < 1 || n_slots > 8 || z_stride_words > 0xffffffffull) return cudaErrorInvalidValue;
+  const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
+  const int n_sl = G.B * G.H;
+  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
+  float* part = scratch + ((n_sl + 63) / 64) * 64;
+  dim3 grid(n_sl, splits, n_slots);
+  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words};
+  for (int i = 0; i < n_slots; ++i) ap.slot_layer[i] = slot_layers[i];
+  decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, slot_layers[0], static_cast<const __nv_bfloat16*>(q), nullptr,
+                                                        part, tickets, status, ap, tm->k, tm->v);
   return cudaGetLastError();
 }
 
@@ -616,7 +657,7 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
   StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                new_len, nullptr, nullptr, 0, 0, {}};
+                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u};
   if (seg_hint) {
     ap.n_seg = G.T + 1;
     for (int l = 0; l <= G.T; ++l) ap.seg[l] = seg_hint[l];
