@@ -47,9 +47,9 @@ def _not_borderline(V, rho):
         assert np.min(np.abs(run - np.round(run))) > 1e-5
 
 
-@pytest.mark.parametrize("dtype,d,t,T,rho,c", [("bf16", 128, 128, 2, 2.0 ** -3.3, 0.75), ("fp32", 64, 64, 1, 2.0 ** -3.3, 0.5),
-                                               ("bf16", 128, 256, 1, 0.0, 0.0)])
-def test_bucketed_append_compress_decode(cuda_lib, dtype, d, t, T, rho, c):
+@pytest.mark.parametrize("dtype,d,t,T,rho,c,W", [("bf16", 128, 128, 2, 2.0 ** -3.3, 0.75, 0), ("fp32", 64, 64, 1, 2.0 ** -3.3, 0.5, 0),
+                                                 ("bf16", 128, 256, 1, 0.0, 0.0, 0), ("bf16", 128, 64, 3, 2.0 ** -3.3, 0.75, 48)])
+def test_bucketed_append_compress_decode(cuda_lib, dtype, d, t, T, rho, c, W):
     B, H, g, nb, i_top = 2, 2, 4, 5, 4
     chunks = [700, 300, 1048]
     n = sum(chunks)
@@ -60,9 +60,10 @@ def test_bucketed_append_compress_decode(cuda_lib, dtype, d, t, T, rho, c):
             K[b, h], V[b, h] = _stream(77, b, h, n, d, dtype, 0.06 if c > 0 else 1.0)
     _not_borderline(V, rho)
     assert math.sqrt(np.max(np.sum(V.astype(np.float64) ** 2, -1))) <= 2.0 ** i_top
-    hz = Harness(cuda_lib, B=B, L=nb + 1, H=H, g=g, d=d, dtype=dtype, t=t, T=T, N=n, seed=11, c_override=c)
+    # W > 0: every instance keeps the newest W tokens of its own sub-stream out of the batches
+    hz = Harness(cuda_lib, B=B, L=nb + 1, H=H, g=g, d=d, dtype=dtype, t=t, T=T, N=n, W=W, seed=11, c_override=c)
     bo = {(b, h): BucketedOracle(d=d, t=t, T=T, i_top=i_top, n_buckets=nb, erase_ratio=rho, layer0=0, head=h,
-                                 max_tokens=n, seed=11 + b, c_override=c) for b in range(B) for h in range(H)}
+                                 max_tokens=n, seed=11 + b, c_override=c, W=W) for b in range(B) for h in range(H)}
     per_slot_events = {}
     p = 0
     for m in chunks:
