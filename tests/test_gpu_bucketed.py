@@ -131,10 +131,13 @@ def test_bucketed_append_compress_decode(cuda_lib, dtype, d, t, T, rho, c, W):
     assert hz.ctx.stats()["device_status"] == 0
 
 
-def test_bucketed_per_stream_entry_and_refusals(cuda_lib):
+@pytest.mark.parametrize("capacity", [500, 300])
+def test_bucketed_per_stream_entry_and_refusals(cuda_lib, capacity):
+    """capacity 500: every instance could take the whole block; capacity 300: only the actual per-bucket
+    counts fit, and repeating the block overflows an instance (refused as a whole)."""
     d, t, n = 128, 64, 500
     ctx = cuda_lib.Context(n_seqs=1, n_layers=4, n_kv_heads=2, n_q_heads=8, head_dim=d, dtype="bf16", block=t, levels=1,
-                           max_tokens=n)
+                           max_tokens=capacity)
     k, v = _stream(78, 0, 1, n, d, "bf16", 1.0)
     _not_borderline(v, 0.0)
     Kd, Vd = to_device(k, "bf16"), to_device(v, "bf16")
@@ -155,6 +158,11 @@ def test_bucketed_per_stream_entry_and_refusals(cuda_lib):
         assert sum(ctx.level_sizes(0, s, 0)) == 0                 # the other head's instances are untouched
     with pytest.raises(Exception):
         ctx.stream_append_bucketed(0, 2, 4, 4, 1, Kd, Vd)         # slots beyond the context's layers
+    if capacity == 300:
+        with pytest.raises(Exception):                            # an instance would overflow: refused, nothing appended
+            for _ in range(3):
+                ctx.stream_append_bucketed(0, 0, 4, 4, 1, Kd, Vd)
+        assert all(sum(ctx.level_sizes(0, s, 1)) <= capacity for s in range(4))
 
 
 def test_bucketed_llama_layer_full_size_sampled_instances(cuda_lib):
