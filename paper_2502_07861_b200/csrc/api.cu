@@ -21,6 +21,7 @@ bool walk_tc_supported(const Geom& G);
 cudaError_t walk_tc_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** tmaps_out);
 void walk_tc_release(void* tmaps);
 bool decode_mma_supported(const Geom& G);
+int decode_mma_ctas_per_sm();
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out);
 void decode_mma_release(void* maps);
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
@@ -34,7 +35,7 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
                                 void* out, int n_heads, int d, cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st);
 }  // namespace bkv
 
 #define BKV_CUDA(expr)                                                                    \
@@ -67,6 +68,7 @@ struct balancekv_ctx {
   int* d_status = nullptr;
   float* d_decode_scratch = nullptr;
   int max_splits = 1;
+  int decode_slots = 148;        // CTAs of the decode kernel that are resident at once
   bool use_tc = false;
   void* tmaps = nullptr;
   void* decode_maps = nullptr;   // tensor maps of the tensor-core decode kernel (bf16, d = 128)
@@ -120,6 +122,13 @@ struct balancekv_ctx {
 
   int64_t tokens_appended = 0, calls_run = 0, kernels_launched = 0;
   std::vector<std::vector<int>> layer_stream_ids;
+
+  // Chain of decode launches: true while the last work this context enqueued was a launch of the
+  // tensor-core decode kernel on chain_stream.  The next decode launch on that stream may then fetch
+  // cache tiles before its grid dependency resolves (only the previous launch can still be running,
+  // and it writes one row per stream).  Every other enqueuing call breaks the chain.
+  bool decode_chain = false;
+  cudaStream_t chain_stream = nullptr;
 
   // value-norm buckets (Algorithm 1): running v_max^2 and the largest erased bucket index, indexed
   // by the stream of the first bucket slot; routing buffers sized for the largest block so far
@@ -330,7 +339,9 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   if (cudaMemset(c->d_fail, 0, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   {
     const int n_sl = f.n_seqs * f.n_kv_heads;
-    c->max_splits = std::max(1, std::min(64, 2 * c->sm_count / n_sl));   // two resident CTAs per SM; rounding down keeps one wave
+    const int per_sm = f.gram_path != 1 && decode_mma_supported(G) ? decode_mma_ctas_per_sm() : 2;
+    c->decode_slots = per_sm * c->sm_count;                                 // CTAs of one wave
+    c->max_splits = std::max(1, std::min(64, c->decode_slots / n_sl));      // rounding down keeps one wave
     if (f.decode_splits > 0) c->max_splits = std::min(64, f.decode_splits);
     const size_t sb = decode_scratch_bytes(G, c->max_splits);
     if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->d_decode_scratch), sb))) return fail(rc);
@@ -397,6 +408,7 @@ static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int le
   if (!K || !V || n < 0) return BALANCEKV_E_INVAL;
   if (!aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
   if (n == 0) return BALANCEKV_OK;
+  c->decode_chain = false;
   const balancekv_config& f = c->cfg;
   const Layout& Lo = c->Lo;
   const int T = Lo.T;
@@ -519,6 +531,7 @@ int balancekv_cache_load_level(balancekv_ctx* c, int layer, int level, const voi
 // level-0 remainder moves and the segment-table update.
 static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
   const Geom& G = c->G;
+  c->decode_chain = false;
   // Every descriptor array of the batch (the calls of each level, the remainder moves, the segment
   // updates) travels in one transfer ahead of the first kernel, so that no copy sits between two
   // kernels of the batch; if they do not fit one half of the ring they go array by array.
@@ -699,8 +712,12 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
     if (c->decode_maps) {
       Seg hint[kMaxLevels + 1];
       const bool alike = layer_seg_hint(c, layer, hint);
+      cudaStream_t st = static_cast<cudaStream_t>(stream);
+      const int early = alike && c->decode_chain && c->chain_stream == st;
       BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                      nullptr, nullptr, 0, 0, 0, alike ? hint : nullptr, static_cast<cudaStream_t>(stream)));
+                                      nullptr, nullptr, 0, 0, 0, alike ? hint : nullptr, early, st));
+      c->decode_chain = true;
+      c->chain_stream = st;
     } else
       BKV_CUDA(launch_decode(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status,
                              static_cast<cudaStream_t>(stream)));
@@ -755,6 +772,7 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
   if (!c || !q || !out || !layers_num || !layers_den || n_num < 1 || n_den < 1) return BALANCEKV_E_INVAL;
   if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
   if (!c->decode_maps) return BALANCEKV_E_INVAL;          // bf16, head_dim 128, group <= 8 only
+  c->decode_chain = false;
   // distinct slots in order of first appearance, with the sides they enter
   int slots[BALANCEKV_MAX_MERGE];
   unsigned num_mask = 0, den_mask = 0;
@@ -788,7 +806,7 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
     c->bytes_resident += block_bytes * BALANCEKV_MAX_MERGE;
   }
   // One launch over all slots (grid z = slot).  The split factor is the largest any slot asks for,
-  // bounded so that the whole grid stays within one wave of two CTAs per SM where it can.
+  // bounded so that the whole grid stays within one wave where it can.
   int splits = 1;
   unsigned keys_mask = 0;
   for (int p = 0; p < n_parts; ++p) {
@@ -796,7 +814,7 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
     if (!((num_mask >> p) & 1u)) keys_mask |= 1u << p;     // a slot that only enters the denominator: values are not read
   }
   const int n_sl = c->cfg.n_seqs * c->cfg.n_kv_heads;
-  splits = std::max(1, std::min(splits, 2 * c->sm_count / std::max(1, n_sl * n_parts)));
+  splits = std::max(1, std::min(splits, c->decode_slots / std::max(1, n_sl * n_parts)));
   {
     ProfScope ps(c, 4, st);
     BKV_CUDA(launch_decode_parts_mma_slots(c->G, c->A, slots, n_parts, keys_mask, q, c->two_acc, c->two_ml, c->two_scratch,
@@ -838,10 +856,13 @@ int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void
         StreamState& S = c->st[s];
         S.len0 += 1; S.appended += 1; S.pending += 1; c->tokens_appended += 1;
       }
-      ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
+      cudaStream_t st = static_cast<cudaStream_t>(stream);
+      const int early = alike && c->decode_chain && c->chain_stream == st;
+      ProfScope ps(c, 4, st);
       BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                      k_new, v_new, rel, idx0, new_len, alike ? hint : nullptr,
-                                      static_cast<cudaStream_t>(stream)));
+                                      k_new, v_new, rel, idx0, new_len, alike ? hint : nullptr, early, st));
+      c->decode_chain = true;
+      c->chain_stream = st;
       c->kernels_launched++;
       return BALANCEKV_OK;
     }
@@ -919,6 +940,7 @@ int balancekv_cache_view(balancekv_ctx* c, int seq, int layer, int kv_head, cons
   if (seq < 0 || seq >= f.n_seqs || layer < 0 || layer >= f.n_layers || kv_head < 0 || kv_head >= f.n_kv_heads)
     return BALANCEKV_E_INVAL;
   BKV_CUDA(cudaDeviceSynchronize());
+  c->decode_chain = false;
   const int s = stream_id(c, seq, layer, kv_head);
   const StreamState& S = c->st[s];
   int64_t total = S.len0;
@@ -1006,6 +1028,7 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
   if (i_top < -60 || i_top > 60 || !(rho >= 0.f) || rho > 1.f) return BALANCEKV_E_INVAL;
   const int n_sl = (int)heads.size();
   if (n_sl < 1) return BALANCEKV_E_INVAL;
+  c->decode_chain = false;
   if (c->bucket_vmax2.empty()) {
     c->bucket_vmax2.assign(c->n_streams, 0.f);
     c->bucket_erase_max.assign(c->n_streams, INT32_MIN);
@@ -1132,6 +1155,7 @@ int balancekv_stream_append_layer_bucketed(balancekv_ctx* c, int layer0, int n_b
 int balancekv_reset(balancekv_ctx* c, void* stream) {
   if (!c) return BALANCEKV_E_INVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->decode_chain = false;
   for (StreamState& S : c->st) S = StreamState();
   c->bucket_vmax2.clear();
   c->bucket_erase_max.clear();

@@ -4,14 +4,15 @@
 //
 // (output ratio of Algorithm 1 / estimator of Theorem 3.3 over the sets C^T..C^0 of a stream;
 // Eq. (1) when every token sits in C^0).  The g <= 8 query heads of a KV head form the rows of a
-// 16-row MMA tile, so q.K^T and p.V each cost one mma.sync.m16n8k16 per 8 tokens x 16 dims: at
-// g = 5 the CUDA-core formulation needs ~65 instructions per token and is issue bound far below
-// HBM speed, this one needs ~6.
+// 8-column MMA operand, so K.q^T and V^T.p^T each cost one mma.sync.m16n8k16 per 16 tokens x 16 dims:
+// at g = 5 the CUDA-core formulation needs ~65 instructions per token and is issue bound far below
+// HBM speed, this one needs ~3.
 //
-// Grid (streams of the layer, splits), 4 warps.  A CTA walks its share of the stream's 64-token
-// tiles through a 3-stage ring filled by TMA (tensor maps over the K and V arenas, boxes of
-// 64 dims x 64 rows, 128-byte swizzle, so ldmatrix reads are bank-conflict free).  Warp w owns
-// tokens 16w..16w+15 of a tile and keeps a private online softmax (running max, sum, 16 x 128
+// Grid (streams of the layer, splits), one CTA of 16 warps in eight groups per SM.  A CTA walks its share of the stream's
+// 64-token tiles through a 6-stage ring filled by TMA (tensor maps over the K and V arenas, boxes of
+// 64 dims x 64 rows, 128-byte swizzle, so ldmatrix reads are bank-conflict free); the groups take
+// tiles in turn.  Warp w of a group owns tokens 32w..32w+31 of a tile -- the tokens are the M
+// dimension of both products -- and keeps a private online softmax (running max, sum, 128 x 8
 // accumulator) in registers; warps merge through shared memory, splits through a global scratch
 // and a ticket counter (the last CTA of a stream combines; nobody waits).
 // Fused decode step: with k_new / v_new given, the launch also appends one token per stream
@@ -29,16 +30,26 @@ namespace bkv {
 
 namespace {
 
-constexpr int kThreads = 128;
-constexpr int kWarps = 4;
+// Shape of a CTA: kGroups warp groups that take the CTA's tiles in turn, each warp of a group owning
+// kTB blocks of 16 tokens of a 64-token tile; kStages tiles in flight; kCtasPerSm resident CTAs.
+constexpr int kGroups = 2;
+constexpr int kTB = 2;
 constexpr int kStages = 3;
+constexpr int kCtasPerSm = 2;
+constexpr int kWarpTokens = 16 * kTB;
+constexpr int kGroupWarps = 64 / kWarpTokens;
+constexpr int kGroupThreads = 32 * kGroupWarps;
+constexpr int kWarps = kGroups * kGroupWarps;
+constexpr int kThreads = 32 * kWarps;
+constexpr int kBars = kGroups * kStages;      // tile i: stage i % kStages, barrier i % kBars (a multiple of kStages and kGroups)
 constexpr int kTN = 64;                      // tokens per tile
 constexpr int kD = 128;
 constexpr uint32_t kHalf = kTN * 128;        // bytes of one [64 tokens][64 dims] bf16 box
 constexpr uint32_t kTensorBytes = 2 * kHalf; // K (or V) tile: two boxes
 constexpr uint32_t kStageBytes = 2 * kTensorBytes;
-constexpr long long kWaitCycles = 4000000000LL;
-constexpr int PS = kD + 4;                   // partial row: acc[D], max, sum, 2 pad (rows stay 16-byte aligned)
+constexpr long long kWaitCycles = 200000000LL;   // about 0.1 s: a bulk copy that has not landed by then never will
+constexpr int kChunks = 1;                   // barriers of the combine's staging copy
+constexpr int PS = kD + 4;                   // row of the in-CTA merge buffer: acc[D], max, sum, 2 pad (bank-conflict free)
 
 struct DecodeMaps {
   CUtensorMap k, v;
@@ -87,6 +98,18 @@ __device__ inline void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t 
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// Transpose of an 8 x 8 matrix of 16-bit elements held one row pair per thread (row lane / 4,
+// columns 2 (lane % 4) and the next): turns C-fragment rows into B-fragment columns.
+__device__ inline uint32_t movm_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ inline float fast_exp2(float x) {     // -inf -> 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ inline uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -121,6 +144,11 @@ struct StepAppend {
   int slot_layer[8];
   unsigned keys_mask;
   unsigned z_stride;
+  // 1: the library's previous launch on this CUDA stream was a decode launch of this context, so
+  // the only arena rows that can still be in flight are the one row per stream that launch
+  // appended.  Every other tile may then be fetched before the grid dependency is resolved (see
+  // the kernel's prologue).  Needs the segment table as a parameter (n_seg > 0).
+  int early;
 };
 
 struct TileRef {
@@ -143,7 +171,20 @@ __device__ inline TileRef locate_tile(int tile, const int* lvl_tiles, const Seg*
   return r;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// Named barrier of one warp group (ids 1, 2; id 0 is __syncthreads) that also votes: true if any
+// of the group's threads passes a true predicate.
+__device__ inline bool group_bar_or(int group, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(group + 1), "r"(kGroupThreads), "r"((uint32_t)pred) : "memory");
+  return r != 0;
+}
+
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
                   float* __restrict__ part_base, unsigned* __restrict__ tickets_base, int* __restrict__ status,
                   const StepAppend ap, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -169,26 +210,48 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   __shared__ int is_last_s;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int group = warp / kGroupWarps, wq = warp % kGroupWarps;   // tile parity served, token quarter of the tile
   const int g = G.g;
   const int sl = blockIdx.x;
   const int seq = sl / G.H, head = sl % G.H;
   const int stream = (seq * G.L + layer) * G.H + head;
   const int splits = gridDim.y, split = blockIdx.y;
   const int64_t stream_base = (int64_t)stream * G.rows_per_stream;
+  // Merge and combine phases: the first work item of this warp, (head mh, way mw) with warp = mw g + mh.
+  int mh = warp, mw = 0;
+  if (g < kWarps)
+    while (mh >= g) { mh -= g; ++mw; }
 
   // Launched with programmatic stream serialization, this grid may become resident while the
-  // previous kernel of the stream is still finishing (the launch latency overlaps its tail);
-  // nothing that kernel wrote is touched before the wait below.  Without the launch attribute
-  // both instructions do nothing.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // previous kernel of the stream is still finishing.  What precedes griddepcontrol.wait touches
+  // nothing that kernel may still write: barrier set-up, and -- in a chain of decode launches
+  // (ap.early) -- the fetch of this CTA's first tiles, except the stream's last tile, which holds the
+  // row the previous step appended.  The dependents are released only after the wait, so at most
+  // one earlier launch of the chain is ever in flight.  Without the launch attribute both
+  // instructions do nothing.
   if (tid == 0) {
-    for (int s = 0; s <= kStages; ++s) mbar_init(&full[s], 1);       // full[kStages]: the combine's bulk copy
+    for (int s = 0; s < kBars + kChunks; ++s) mbar_init(&full[s], 1);     // full[kBars ..]: the combine's staging copies
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // The step's operands are wanted right after the dependency resolves: ask for them in L2 now.  A
+  // line fetched before its producer has written it is harmless, L2 being the point of coherence
+  // (the producer's write updates that line; nothing is taken into L1 here).
+  if (tid < 2 * g) {
+    const char* qrow = reinterpret_cast<const char*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + (tid >> 1)) * kD);
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(qrow + 128 * (tid & 1)));
+  } else if (ap.k_new && tid < 2 * g + 4) {
+    const int k = tid - 2 * g;
+    const char* row = reinterpret_cast<const char*>((k & 2 ? ap.v_new : ap.k_new) + (size_t)sl * kD);
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(row + 128 * (k & 1)));
+  }
+  const bool early = ap.early && ap.n_seg;
+  if (!early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   if (tid <= G.T) {
     const Seg s = ap.n_seg ? ap.seg[tid] : A.seg[(size_t)stream * (G.T + 1) + tid];
     seg_s[tid] = s;
@@ -201,10 +264,10 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const int t_end = (int)((long long)n_tiles * (split + 1) / splits);
   const int my_tiles = t_end - t_begin;
 
-  auto issue = [&](int i) {   // thread 0 only
+  auto issue = [&](int i) {   // one thread
     const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
     unsigned char* st = tiles + (size_t)(i % kStages) * kStageBytes;
-    uint64_t* bar = &full[i % kStages];
+    uint64_t* bar = &full[i % kBars];
     mbar_expect_tx(bar, keys_only ? kTensorBytes : kStageBytes);
     tma_load_2d(st, &tmK, 0, (int)tr.row, bar);
     tma_load_2d(st + kHalf, &tmK, 64, (int)tr.row, bar);
@@ -213,171 +276,334 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       tma_load_2d(st + kTensorBytes + kHalf, &tmV, 64, (int)tr.row, bar);
     }
   };
-  if (tid == 0)
-    for (int i = 0; i < min(kStages, my_tiles); ++i) issue(i);
+  int issued = 0;
+  if (tid == 0) {
+    const int lim = min(kStages, my_tiles);
+    while (issued < lim && !(early && t_begin + issued == n_tiles - 1)) issue(issued++);
+  }
+  if (early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid == 0)
+      while (issued < min(kStages, my_tiles)) issue(issued++);
+  }
 
-  // A fragments of the query tile: row = query head of the group (rows >= g are zero)
-  const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-  uint32_t qa[8][4];
+  // B fragments of the query tile (k = dims, n = query head of the group; heads >= g are zero).
+  // The tokens are the M dimension of both products (S^T = K Q^T, O^T = V^T P^T), so a warp spends
+  // one mma.sync.m16n8k16 per 16 tokens x 16 dims instead of the two that a query-major tile
+  // (16 rows, at most 8 of them used) needs.
+  const int hq = lane >> 2, tq = lane & 3;         // C fragment: rows hq, hq + 8; columns 2 tq, 2 tq + 1
+  uint32_t qb[8][2];
   {
-    const __nv_bfloat16* qp = q + ((size_t)seq * (G.H * g) + (size_t)head * g + qrow) * kD;
+    const __nv_bfloat16* qp = q + ((size_t)seq * (G.H * g) + (size_t)head * g + hq) * kD;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       uint32_t lo = 0, hi = 0;
-      if (qrow < g) {
-        lo = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + qcol);
-        hi = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + qcol);
+      if (hq < g) {
+        lo = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 2 * tq);
+        hi = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * tq);
       }
-      qa[ks][0] = lo; qa[ks][1] = 0; qa[ks][2] = hi; qa[ks][3] = 0;
+      qb[ks][0] = lo; qb[ks][1] = hi;
     }
   }
   const float sc = 1.4426950408889634f * G.inv_sqrt_d;
 
-  float o[16][4];
+  // O^T of this warp's tokens: o[mb][j] = dim 16 mb + hq + 8 (j >> 1), query head 2 tq + (j & 1)
+  float o[8][4];
 #pragma unroll
-  for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-  float m_run = -INFINITY, l_run = 0.f;      // of row qrow, over this thread's columns
+  for (int n = 0; n < 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads 2 tq, 2 tq + 1; l over this thread's tokens
 
-  // ldmatrix row addresses of this lane (see the fragment layouts of mma.m16n8k16)
+  // ldmatrix row addresses of this lane (see the fragment layouts of mma.m16n8k16), for the first of
+  // the warp's kTB 16-token blocks
   const int mi = lane >> 3, mr = lane & 7;
-  const int k_tok = warp * 16 + (mi >> 1) * 8 + mr, k_chunk = mi & 1;     // K: x4 = (tok 0-7 | 8-15) x (dims lo | hi)
-  const int v_tok = warp * 16 + (mi & 1) * 8 + mr, v_chunk = mi >> 1;     // V (transposed): x4 = (dims lo | hi) x (tok 0-7 | 8-15)
+  const int k_tok = wq * kWarpTokens + (mi & 1) * 8 + mr, k_chunk = mi >> 1;     // K (A operand): x4 = (tok 0-7 | 8-15) x (dims lo | hi)
+  const int v_tok = wq * kWarpTokens + (mi >> 1) * 8 + mr, v_chunk = mi & 1;     // V (A operand, transposed): x4 = (dims lo | hi) x (tok 0-7 | 8-15)
 
+  // The warp groups take tiles in turn (one group: every tile).  With the tiles already in shared
+  // memory the loop is bound by the latency of its dependency chain (barrier, score MMAs, softmax
+  // shuffles, value MMAs).  Tile i lives in stage i % kStages whichever group consumes it; the
+  // group that frees a stage refills it.
   bool failed = false;
-  for (int i = 0; i < my_tiles; ++i) {
+  for (int i = group; i < my_tiles; i += kGroups) {
     const int s = i % kStages;
-    const bool arrived = __all_sync(0xffffffffu, mbar_wait(&full[s], (uint32_t)((i / kStages) & 1)));
+    // Barrier i % kBars serves tiles i, i + kBars, ... only, all of them this group's: the phase
+    // before the awaited one is a tile the group has consumed itself, so the parity wait cannot be
+    // a phase off although the groups advance independently.  One lane polls (every poll of a
+    // barrier is a serialised shared-memory access).
+    bool arrived = true;
+    if (lane == 0) arrived = mbar_wait(&full[i % kBars], (uint32_t)((i / kBars) & 1));
+    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+    __syncwarp();                  // the polling lane's view of the landed tile, for the whole warp
     const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
     const uint32_t Kt = smem_u32(tiles + (size_t)s * kStageBytes), Vt = Kt + kTensorBytes;
-    if (arrived && warp * 16 < tr.rows) {
-      // ---- scores of the 16 tokens of this warp: S[16 x 16] = Q K^T
-      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    if (arrived && wq * kWarpTokens < tr.rows) {
+      // ---- scores of the warp's tokens against the group's heads: S^T[16 x 8] = K Q^T per block.
+      // A dependent mma.sync waits for its predecessor's whole latency and the asm statements keep
+      // their order: operand loads go first, and the MMAs form 4 chains per block issued in turn.
+      float sa[kTB][4][4];
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        uint32_t kb[4];
-        ldsm_x4(Kt + tile_off(k_tok, ks * 2 + k_chunk), kb);
-        mma_bf16(s0, qa[ks], kb[0], kb[1]);
-        mma_bf16(s1, qa[ks], kb[2], kb[3]);
+      for (int tb = 0; tb < kTB; ++tb)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { sa[tb][c][0] = sa[tb][c][1] = sa[tb][c][2] = sa[tb][c][3] = 0.f; }
+#pragma unroll
+      for (int kh = 0; kh < 2; ++kh) {
+        uint32_t ka[4][kTB][4];
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+#pragma unroll
+          for (int tb = 0; tb < kTB; ++tb) ldsm_x4(Kt + tile_off(k_tok + 16 * tb, (kh * 4 + k4) * 2 + k_chunk), ka[k4][tb]);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+#pragma unroll
+          for (int tb = 0; tb < kTB; ++tb) mma_bf16(sa[tb][k4], ka[k4][tb], qb[kh * 4 + k4][0], qb[kh * 4 + k4][1]);
       }
-      // this thread: row qrow, tokens tcol, tcol+1 (s0) and tcol+8, tcol+9 (s1)
-      const int tcol = warp * 16 + qcol;
+      // the value operands do not depend on the probabilities: their loads are in flight during the softmax
+      uint32_t va[kTB][8][4];
+      if (!keys_only) {
+#pragma unroll
+        for (int tb = 0; tb < kTB; ++tb)
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) ldsm_x4_trans(Vt + tile_off(v_tok + 16 * tb, mb * 2 + v_chunk), va[tb][mb]);
+      }
+      // this thread: per block tb the tokens tok0 (x[tb][0], x[tb][1]) and tok0 + 8 (x[tb][2], x[tb][3]),
+      // heads 2 tq (even index) and 2 tq + 1
       const float lvl = (float)tr.level;
-      float x0 = tcol < tr.rows ? fmaf(s0[0], sc, lvl) : -INFINITY;
-      float x1 = tcol + 1 < tr.rows ? fmaf(s0[1], sc, lvl) : -INFINITY;
-      float x2 = tcol + 8 < tr.rows ? fmaf(s1[0], sc, lvl) : -INFINITY;
-      float x3 = tcol + 9 < tr.rows ? fmaf(s1[1], sc, lvl) : -INFINITY;
-      float mx = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(m_run, mx);                   // finite: token 16 w of the tile is valid
-      if (__any_sync(0xffffffffu, m_new > m_run)) {
-        const float a = exp2f(m_run - m_new);                 // m_run = -inf -> 0
-        l_run *= a;
+      float x[kTB][4];
+      float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-        for (int n = 0; n < 16; ++n) { o[n][0] *= a; o[n][1] *= a; }
-        m_run = m_new;
+      for (int tb = 0; tb < kTB; ++tb) {
+        const int tok0 = wq * kWarpTokens + tb * 16 + hq;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          x[tb][j] = tok0 + 8 * (j >> 1) < tr.rows
+                         ? fmaf((sa[tb][0][j] + sa[tb][1][j]) + (sa[tb][2][j] + sa[tb][3][j]), sc, lvl) : -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(x[tb][0], x[tb][2]));
+        mx1 = fmaxf(mx1, fmaxf(x[tb][1], x[tb][3]));
       }
-      x0 = exp2f(x0 - m_run); x1 = exp2f(x1 - m_run); x2 = exp2f(x2 - m_run); x3 = exp2f(x3 - m_run);
-      l_run += (x0 + x1) + (x2 + x3);
-      // the probabilities enter the second MMA as bf16: split them into a high and a low part
-      // (p = hi + lo to 16 bits) so that the output error stays that of the final rounding
-      const uint32_t ph[4] = {pack_bf16(x0, x1), 0u, pack_bf16(x2, x3), 0u};
-      const uint32_t pl[4] = {pack_bf16(x0 - bf16_lo(ph[0]), x1 - bf16_hi(ph[0])), 0u,
-                              pack_bf16(x2 - bf16_lo(ph[2]), x3 - bf16_hi(ph[2])), 0u};
-      // ---- O[16 x 128] += P[16 x 16] V[16 x 128]
-      if (!keys_only)
 #pragma unroll
-      for (int nb = 0; nb < 8; ++nb) {
-        uint32_t vb[4];
-        ldsm_x4_trans(Vt + tile_off(v_tok, nb * 2 + v_chunk), vb);
-        mma_bf16(o[2 * nb], ph, vb[0], vb[1]);
-        mma_bf16(o[2 * nb], pl, vb[0], vb[1]);
-        mma_bf16(o[2 * nb + 1], ph, vb[2], vb[3]);
-        mma_bf16(o[2 * nb + 1], pl, vb[2], vb[3]);
+      for (int off = 4; off < 32; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+      }
+      const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite: the warp's first token of the tile is valid
+      if (__any_sync(0xffffffffu, mn0 > m_run[0] || mn1 > m_run[1])) {
+        const float a0 = fast_exp2(m_run[0] - mn0), a1 = fast_exp2(m_run[1] - mn1);   // m_run = -inf -> 0
+        l_run[0] *= a0; l_run[1] *= a1;
+#pragma unroll
+        for (int n = 0; n < 8; ++n) { o[n][0] *= a0; o[n][1] *= a1; o[n][2] *= a0; o[n][3] *= a1; }
+        m_run[0] = mn0; m_run[1] = mn1;
+      }
+      // The probabilities enter the second MMA as bf16: split them into a high and a low part
+      // (p = hi + lo to 16 bits) so that the output error stays that of the final rounding.  Each
+      // packed register is a row of an 8 x 8 [token][head] matrix; the B operand wants [head][token].
+      uint32_t bh[kTB][2], bl[kTB][2];
+#pragma unroll
+      for (int tb = 0; tb < kTB; ++tb) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[tb][j] = fast_exp2(x[tb][j] - m_run[j & 1]);
+        l_run[0] += x[tb][0] + x[tb][2];
+        l_run[1] += x[tb][1] + x[tb][3];
+        const uint32_t ph0 = pack_bf16(x[tb][0], x[tb][1]), ph1 = pack_bf16(x[tb][2], x[tb][3]);
+        const uint32_t pl0 = pack_bf16(x[tb][0] - bf16_lo(ph0), x[tb][1] - bf16_hi(ph0));
+        const uint32_t pl1 = pack_bf16(x[tb][2] - bf16_lo(ph1), x[tb][3] - bf16_hi(ph1));
+        bh[tb][0] = movm_trans(ph0); bh[tb][1] = movm_trans(ph1);
+        bl[tb][0] = movm_trans(pl0); bl[tb][1] = movm_trans(pl1);
+      }
+      // ---- O^T[128 x 8] += V^T[128 x 16 kTB] P^T[16 kTB x 8]: the high parts of a block, then its low
+      // parts, so that no MMA follows its predecessor on the same accumulator
+      if (!keys_only) {
+#pragma unroll
+        for (int tb = 0; tb < kTB; ++tb) {
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bh[tb][0], bh[tb][1]);
+#pragma unroll
+          for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bl[tb][0], bl[tb][1]);
+        }
       }
     }
-    // stage s fully consumed; the same barrier makes a timed-out wait a CTA-wide decision
-    if (__syncthreads_or(!arrived)) { failed = true; break; }
-    if (tid == 0 && i + kStages < my_tiles) issue(i + kStages);
+    // the group has consumed stage s; the same barrier makes a timed-out wait a group-wide decision
+    if (group_bar_or(group, !arrived)) { failed = true; break; }
+    if (tid == group * kGroupThreads && i + kStages < my_tiles) issue(i + kStages);
   }
-  if (failed && tid == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
-  __syncthreads();
+  if (failed && lane == 0 && wq == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
 
-  // ---- merge the 4 warps through shared memory (the tile ring is idle now)
+  // ---- merge the warps through shared memory (after the barrier the tile ring is idle)
   float* mrg = reinterpret_cast<float*>(tiles);        // [kWarps][g][PS]
-  {
-    float l = l_run;
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (qrow < g) {
-      float* rowp = mrg + ((size_t)warp * g + qrow) * PS;
 #pragma unroll
-      for (int n = 0; n < 16; ++n) { rowp[n * 8 + qcol] = o[n][0]; rowp[n * 8 + qcol + 1] = o[n][1]; }
-      if ((lane & 3) == 0) { rowp[kD] = m_run; rowp[kD + 1] = l; }
+  for (int off = 4; off < 32; off <<= 1) {
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int h = 2 * tq + e;
+    if (h < g) {
+      float* rowp = mrg + ((size_t)warp * g + h) * PS;
+#pragma unroll
+      for (int n = 0; n < 8; ++n) { rowp[16 * n + hq] = o[n][e]; rowp[16 * n + 8 + hq] = o[n][2 + e]; }
+      if (hq == 0) { rowp[kD] = m_run[e]; rowp[kD + 1] = l_run[e]; }
     }
   }
   __syncthreads();
   // With a single split the CTA's partial is the stream's result: it stays in shared memory (behind
-  // the merge buffer) and the ticket, the fences and the staging copy are skipped.
-  constexpr uint32_t kSingleOff = 32768;
+  // the merge buffers) and the ticket, the fences and the staging copy are skipped.
+  constexpr uint32_t kMrg2Off = kWarps * kMaxGroup * PS * 4;        // behind mrg: [ways][g][PS] first-level merges
+  constexpr uint32_t kSingleOff = kMrg2Off + kWarps * PS * 4 + 512;
   const bool single = splits == 1;
-  float* my_part = single ? reinterpret_cast<float*>(tiles + kSingleOff) : part + ((size_t)sl * splits + split) * g * PS;
-  for (int i = tid; i < g * kD; i += kThreads) {
-    const int h = i / kD, c = i % kD;
-    float M = -INFINITY;
+  // Partial results: per (stream, split, head) a row of kD column sums, and behind all rows the
+  // (max, sum) pairs.  Rows of 512 bytes keep the staging copy 128-byte aligned.
+  const size_t n_rows_all = (size_t)gridDim.x * splits * g;
+  float* my_acc = single ? reinterpret_cast<float*>(tiles + kSingleOff) : part + ((size_t)sl * splits + split) * g * kD;
+  float* my_ml = single ? reinterpret_cast<float*>(tiles + kSingleOff) + kMaxGroup * kD
+                        : part + n_rows_all * kD + ((size_t)sl * splits + split) * g * 2;
+  // Work items of the merge and combine phases: (head mh, way mw), item r = mw g + mh, ways =
+  // max(1, warps / g); a warp takes items r = warp, warp + kWarps, ... (lane = 4 output columns).
+  // The ways of a head share its rows: way mw takes the rows mw, mw + ways, ...
+  const int ways = g >= kWarps ? 1 : kWarps / g;
+  const int n_r = g * ways;
+  if (ways > 1) {
+    // two levels, so that no thread walks all warps' rows
+    float* mrg2 = reinterpret_cast<float*>(tiles + kMrg2Off);
+    if (warp < n_r) {
+      float mv[kWarps], M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mrg[((size_t)w * g + h) * PS + kD]);
-    float acc = 0.f, L = 0.f;
+      for (int k = 0; k < kWarps; ++k) {
+        const int w = mw + k * ways;
+        mv[k] = w < kWarps ? mrg[((size_t)w * g + mh) * PS + kD] : -INFINITY;
+        M = fmaxf(M, mv[k]);
+      }
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float L = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const float* rowp = mrg + ((size_t)w * g + h) * PS;
-      const float f = rowp[kD] == -INFINITY ? 0.f : exp2f(rowp[kD] - M);
-      acc = fmaf(rowp[c], f, acc);
-      L = fmaf(rowp[kD + 1], f, L);
+      for (int k = 0; k < kWarps; ++k) {
+        const int w = mw + k * ways;
+        if (w < kWarps && mv[k] != -INFINITY) {
+          const float* rowp = mrg + ((size_t)w * g + mh) * PS;
+          const float f = fast_exp2(mv[k] - M);
+          const float4 v = *reinterpret_cast<const float4*>(rowp + 4 * lane);
+          acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y); acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+          L = fmaf(rowp[kD + 1], f, L);
+        }
+      }
+      float* dst = mrg2 + ((size_t)mw * g + mh) * PS;
+      *reinterpret_cast<float4*>(dst + 4 * lane) = acc;
+      if (lane == 0) { dst[kD] = M; dst[kD + 1] = L; }
     }
-    my_part[h * PS + c] = acc;
-    if (c == 0) { my_part[h * PS + kD] = M; my_part[h * PS + kD + 1] = L; }
+    __syncthreads();
+    mrg = mrg2;                                 // the second level reads `ways` rows per head
+  }
+  {
+    const int n_src = ways > 1 ? ways : kWarps;
+    for (int h = warp; h < g; h += kWarps) {
+      float M = -INFINITY;
+      for (int k = 0; k < n_src; ++k) M = fmaxf(M, mrg[((size_t)k * g + h) * PS + kD]);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float L = 0.f;
+      for (int k = 0; k < n_src; ++k) {
+        const float* rowp = mrg + ((size_t)k * g + h) * PS;
+        const float mk = rowp[kD];
+        const float f = mk == -INFINITY ? 0.f : fast_exp2(mk - M);
+        const float4 v = *reinterpret_cast<const float4*>(rowp + 4 * lane);
+        acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y); acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+        L = fmaf(rowp[kD + 1], f, L);
+      }
+      *reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane) = acc;
+      if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
+    }
   }
   // ---- ticket: the last CTA of the stream combines the splits
   if (!single) {
-    __threadfence();
+    // release / acquire through one thread: the barrier orders the CTA's writes before thread 0's
+    // fence and its fence after the ticket before everybody's reads (fences are cumulative); a
+    // fence by every thread costs a microsecond here
     __syncthreads();
     if (tid == 0) {
+      __threadfence();
       const unsigned old = atomicAdd(&tickets[sl], 1u);
       is_last_s = old == (unsigned)(splits - 1);
+      if (is_last_s) __threadfence();
     }
     __syncthreads();
     if (!is_last_s) return;
-    __threadfence();
   } else {
     __syncthreads();
   }
-  // Combine: first the (max, sum) pairs of all splits in one round of loads, then every thread
-  // sums its output columns over the splits with independent loads.
-  const float* sp = part + (size_t)sl * splits * g * PS;   // 16-byte aligned: rows of PS * 4 = 528 bytes
+  // Combine.  All partial rows of the stream are contiguous; if they fit, one bulk copy brings them
+  // into the idle tile ring, otherwise they are read from global memory.  The (max, sum) pairs of
+  // all splits are read straight from L2 meanwhile and turned into the scale factors of the splits.
+  // Every global load of this phase is issued before the first of them is consumed: the CTA is
+  // alone on the critical path here, and each dependent round trip would show.
+  const float* sp = part + (size_t)sl * splits * g * kD;
+  const float* sp_ml = single ? my_ml : part + n_rows_all * kD + (size_t)sl * splits * g * 2;
   float* cm = reinterpret_cast<float*>(tiles);            // [splits][g] max, later the scale factors
   float* cl = cm + 64 * kMaxGroup;                        // [splits][g] sums
   float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
   float* cL = cM + kMaxGroup;                             // [g] overall sum
   float* cN = cL + kMaxGroup;                             // [g] factor of the appended token
-  // All partial rows of the stream are contiguous.  If they fit, one bulk copy brings them into
-  // the idle tile ring (a single round trip); otherwise they are read from global memory.
-  constexpr uint32_t kStageOff = 8192;                     // behind cm, cl, cM, cL, cN
-  const uint32_t part_bytes = (uint32_t)splits * g * PS * sizeof(float);
+  float4* red = reinterpret_cast<float4*>(tiles + 4352);  // [ways - 1][g][32] partial column sums (<= 7680 bytes)
+  constexpr uint32_t kStageOff = 16384;                    // behind cm, cl, cM, cL, cN, red
+  const uint32_t part_bytes = (uint32_t)splits * g * kD * sizeof(float);
   const bool staged = single || part_bytes <= kStages * kStageBytes - kStageOff;
   const float* sp_s = reinterpret_cast<const float*>(tiles + (single ? kSingleOff : kStageOff));
+  uint64_t* cbar = full + kBars;
+  if (staged && !single && tid == kThreads - 32) {
+    // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
+    // (acquired above) come before the async-proxy copy
+    asm volatile("fence.proxy.async;" ::: "memory");
+    mbar_expect_tx(cbar, part_bytes);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(tiles + kStageOff)), "l"(sp), "r"(part_bytes), "r"(smem_u32(cbar)) : "memory");
+  }
+  // ---- loads: (max, sum) pairs; the appended token's rows (last warp) and, per lane, 4 dims of k_new
+  // and of q and 4 columns of v_new for this warp's heads
+  constexpr int kMlPer = (64 * kMaxGroup + kThreads - 1) / kThreads;
+  constexpr int kHeadsPer = (kMaxGroup + kWarps - 1) / kWarps;
+  float2 mlv[kMlPer];
+#pragma unroll
+  for (int k = 0; k < kMlPer; ++k) {
+    const int i = tid + k * kThreads;
+    mlv[k] = make_float2(-INFINITY, 0.f);
+    if (i < splits * g) {
+      const float2* mlp = reinterpret_cast<const float2*>(sp_ml) + i;
+      mlv[k] = single ? *mlp : __ldcg(mlp);
+    }
+  }
+  const size_t dst_row = (size_t)stream_base + G.region_off[0] + ap.rel_row;
+  uint4 row_new = make_uint4(0u, 0u, 0u, 0u);
+  uint2 kn = make_uint2(0u, 0u), qv[kHeadsPer], vn_pre = make_uint2(0u, 0u);
+  if (ap.k_new) {
+    if (warp == kWarps - 1)                                   // lanes 0-15: the row of K, lanes 16-31: the row of V
+      row_new = reinterpret_cast<const uint4*>((lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD)[lane & 15];
+    if (warp < g) {
+      kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
+      vn_pre = *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + 4 * lane);
+#pragma unroll
+      for (int k = 0; k < kHeadsPer; ++k) {
+        const int h = warp + k * kWarps;
+        qv[k] = h < g ? *reinterpret_cast<const uint2*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane)
+                      : make_uint2(0u, 0u);
+      }
+    }
+  }
+  // ---- consume
+#pragma unroll
+  for (int k = 0; k < kMlPer; ++k) {
+    const int i = tid + k * kThreads;
+    if (i < splits * g) { cm[i] = mlv[k].x; cl[i] = mlv[k].y; }
+  }
+  float x_new[kHeadsPer];
+#pragma unroll
+  for (int k = 0; k < kHeadsPer; ++k) x_new[k] = 0.f;
   if (ap.k_new) {
     // append (every CTA of the stream has taken its ticket, so nobody reads the old segment table
-    // any more): one 256-byte row of K and of V, the position, the new length of C^0.  Done first,
-    // so that the writes drain while the partials are combined.
-    const size_t dst_row = (size_t)stream_base + G.region_off[0] + ap.rel_row;
-    if (warp == 0) {                                          // lanes 0-15: the row of K, lanes 16-31: the row of V
-      const __nv_bfloat16* src = (lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD;
+    // any more): one 256-byte row of K and of V, the position, the new length of C^0.
+    if (warp == kWarps - 1) {
       __nv_bfloat16* dstp = static_cast<__nv_bfloat16*>(lane < 16 ? A.K : A.V) + dst_row * kD;
-      const uint4 v = reinterpret_cast<const uint4*>(src)[lane & 15];
-      reinterpret_cast<uint4*>(dstp)[lane & 15] = v;
+      reinterpret_cast<uint4*>(dstp)[lane & 15] = row_new;
       float s2 = 0.f;                                         // ||k||^2 / ||v||^2 travel with the row
-      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&row_new);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float2 f = __bfloat1622float2(h2[i]);
@@ -388,143 +614,128 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       for (int o = 8; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
       const float v2 = __shfl_sync(0xffffffffu, s2, 16);
       if (lane == 0 && A.nrm) A.nrm[dst_row] = make_float2(s2, v2);
-    } else if (tid == 32) {
-      A.idx[dst_row] = ap.idx0;
-      A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
-    }
-  }
-  // the appended token's operands are requested now, so that their latency overlaps the staging:
-  // per lane 4 dims of <q_h, k_new> for this warp's (up to two) heads, and this thread's first
-  // four columns of v_new
-  float dot_pre[2] = {0.f, 0.f};
-  uint2 vn_pre = make_uint2(0u, 0u);
-  if (ap.k_new) {
-    const uint2 kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
-    const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&kn.y);
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int h = warp + kWarps * hh;
-      if (h < g) {
-        const uint2 qv = *reinterpret_cast<const uint2*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane);
-        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv.y);
-        float d = __bfloat162float(q01.x) * __bfloat162float(k01.x);
-        d = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), d);
-        d = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), d);
-        d = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), d);
-        dot_pre[hh] = d;
+      if (lane == 1) {
+        A.idx[dst_row] = ap.idx0;
+        A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
       }
     }
-    if (tid < g * (kD / 4)) vn_pre = *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + (tid % (kD / 4)) * 4);
-  }
-  if (staged && !single) {
-    if (tid == 0) {
-      // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
-      // (acquired above) come before the async-proxy copy
-      asm volatile("fence.proxy.async;" ::: "memory");
-      mbar_expect_tx(&full[kStages], part_bytes);
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(tiles + kStageOff)), "l"(sp), "r"(part_bytes), "r"(smem_u32(&full[kStages])) : "memory");
+    if (warp < g) {
+      // the appended token: level 0, weight 1; <q, k_new> in fp32, 4 dims per lane
+      const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&kn.y);
+#pragma unroll
+      for (int k = 0; k < kHeadsPer; ++k) {
+        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv[k].x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv[k].y);
+        float dot = __bfloat162float(q01.x) * __bfloat162float(k01.x);
+        dot = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), dot);
+        dot = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), dot);
+        dot = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), dot);
+        x_new[k] = warp_sum(dot) * sc;
+      }
     }
-    const bool landed = mbar_wait(&full[kStages], 0u);
-    if (__syncthreads_or(!landed)) {
-      if (tid == 0) { atomicCAS(status, kStatusOk, kStatusWaitTimeout); tickets[sl] = 0; }
-      return;
-    }
-  }
-  if (staged) sp = sp_s;
-  for (int i = tid; i < splits * g; i += kThreads) {
-    const float* rowp = sp + (size_t)i * PS;
-    cm[i] = staged ? rowp[kD] : __ldcg(rowp + kD);
-    cl[i] = staged ? rowp[kD + 1] : __ldcg(rowp + kD + 1);
   }
   __syncthreads();
-  for (int h = warp; h < g; h += kWarps) {     // one warp per head, lanes over the (<= 64) splits
+#pragma unroll
+  for (int k = 0; k < kHeadsPer; ++k) {        // one warp per head, lanes over the (<= 64) splits
+    const int h = warp + k * kWarps;
+    if (h >= g) break;
     const int s0 = lane, s1 = lane + 32;
     const float m0 = s0 < splits ? cm[s0 * g + h] : -INFINITY, m1 = s1 < splits ? cm[s1 * g + h] : -INFINITY;
-    const float M = warp_max(fmaxf(m0, m1));
-    const float f0 = m0 == -INFINITY ? 0.f : exp2f(m0 - M), f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M);
-    float L = (s0 < splits ? cl[s0 * g + h] * f0 : 0.f) + (s1 < splits ? cl[s1 * g + h] * f1 : 0.f);
-    L = warp_sum(L);
-    if (!ap.k_new) {
-      if (s0 < splits) cm[s0 * g + h] = f0;
-      if (s1 < splits) cm[s1 * g + h] = f1;
-    }
+    float M = warp_max(fmaxf(m0, m1));
     float fN = 0.f;
-    if (ap.k_new) {
-      // the appended token: level 0, weight 1; <q, k_new> in fp32, 4 dims per lane
-      const float x = warp_sum(h < kWarps ? dot_pre[0] : dot_pre[1]) * sc;
-      const float M2 = fmaxf(M, x);
-      const float fS = M == -INFINITY ? 0.f : exp2f(M - M2);
-      fN = exp2f(x - M2);
-      if (s0 < splits) cm[s0 * g + h] = f0 * fS;
-      if (s1 < splits) cm[s1 * g + h] = f1 * fS;
-      if (lane == 0) { cM[h] = M2; cL[h] = fmaf(L, fS, fN); cN[h] = fN; }
-    } else if (lane == 0) {
-      cM[h] = M; cL[h] = L;
-    }
+    if (ap.k_new) { M = fmaxf(M, x_new[k]); fN = fast_exp2(x_new[k] - M); }
+    const float f0 = m0 == -INFINITY ? 0.f : fast_exp2(m0 - M), f1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - M);
+    float L = (s0 < splits ? cl[s0 * g + h] * f0 : 0.f) + (s1 < splits ? cl[s1 * g + h] * f1 : 0.f);
+    L = warp_sum(L) + fN;
+    if (s0 < splits) cm[s0 * g + h] = f0;
+    if (s1 < splits) cm[s1 * g + h] = f1;
+    if (lane == 0) { cM[h] = M; cL[h] = L; cN[h] = fN; }
   }
   __syncthreads();
-  // every thread owns 4 consecutive output columns of one head; 8 splits' loads in flight
-  const int n_items = g * (kD / 4);
-  for (int i = tid; i < n_items; i += kThreads) {
-    const int h = i / (kD / 4), c = (i % (kD / 4)) * 4;
+  // Column sums over the splits: item (mh, mw) takes the splits mw, mw + ways, ... of its head, lane =
+  // 4 consecutive columns; the ways meet in shared memory.
+  float4 accs[kHeadsPer];
+  bool landed = true;
+  if (staged && !single) {
+    if (lane == 0) landed = mbar_wait(cbar, 0u);
+    landed = __shfl_sync(0xffffffffu, landed, 0);
+    __syncwarp();
+  }
+#pragma unroll
+  for (int k = 0; k < kHeadsPer; ++k) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (staged) {
-      // partial rows in shared memory: plain shared loads, four independent accumulators
-      const float* base = sp_s + (size_t)h * PS + c;
-      const float* fac = cm + h;
-      float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
-      int s = 0;
-      for (; s + 4 <= splits; s += 4) {
-        const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)(s + 0) * g * PS);
-        const float4 v1 = *reinterpret_cast<const float4*>(base + (size_t)(s + 1) * g * PS);
-        const float4 v2 = *reinterpret_cast<const float4*>(base + (size_t)(s + 2) * g * PS);
-        const float4 v3 = *reinterpret_cast<const float4*>(base + (size_t)(s + 3) * g * PS);
-        const float f0 = fac[(s + 0) * g], f1 = fac[(s + 1) * g], f2 = fac[(s + 2) * g], f3 = fac[(s + 3) * g];
-        a0.x = fmaf(v0.x, f0, a0.x); a0.y = fmaf(v0.y, f0, a0.y); a0.z = fmaf(v0.z, f0, a0.z); a0.w = fmaf(v0.w, f0, a0.w);
-        a1.x = fmaf(v1.x, f1, a1.x); a1.y = fmaf(v1.y, f1, a1.y); a1.z = fmaf(v1.z, f1, a1.z); a1.w = fmaf(v1.w, f1, a1.w);
-        a2.x = fmaf(v2.x, f2, a2.x); a2.y = fmaf(v2.y, f2, a2.y); a2.z = fmaf(v2.z, f2, a2.z); a2.w = fmaf(v2.w, f2, a2.w);
-        a3.x = fmaf(v3.x, f3, a3.x); a3.y = fmaf(v3.y, f3, a3.y); a3.z = fmaf(v3.z, f3, a3.z); a3.w = fmaf(v3.w, f3, a3.w);
-      }
-      for (; s < splits; ++s) {
-        const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)s * g * PS);
-        const float f0 = fac[s * g];
-        a0.x = fmaf(v0.x, f0, a0.x); a0.y = fmaf(v0.y, f0, a0.y); a0.z = fmaf(v0.z, f0, a0.z); a0.w = fmaf(v0.w, f0, a0.w);
-      }
-      acc.x = (a0.x + a1.x) + (a2.x + a3.x); acc.y = (a0.y + a1.y) + (a2.y + a3.y);
-      acc.z = (a0.z + a1.z) + (a2.z + a3.z); acc.w = (a0.w + a1.w) + (a2.w + a3.w);
-    } else {
-      for (int s = 0; s < splits; s += 8) {
-        float4 v[8];
+    const int r = warp + k * kWarps;
+    if (r < n_r) {
+      int ih = mh, iw = mw;
+      if (k > 0) { ih = r; iw = 0; }            // more heads than warps: ways = 1
+      const size_t row_stride = (size_t)g * kD, step = (size_t)ways * row_stride;
+      const float* fac = cm + ih + iw * g;
+      const int fstep = ways * g;
+      int n = iw < splits ? (splits - iw + ways - 1) / ways : 0;     // splits of this way
+      if (staged) {
+        const float* p = sp_s + (size_t)iw * row_stride + (size_t)ih * kD + 4 * lane;
+        for (; n >= 4; n -= 4, p += 4 * step, fac += 4 * fstep) {
+          const float4 v0 = *reinterpret_cast<const float4*>(p), v1 = *reinterpret_cast<const float4*>(p + step);
+          const float4 v2 = *reinterpret_cast<const float4*>(p + 2 * step), v3 = *reinterpret_cast<const float4*>(p + 3 * step);
+          const float f0 = fac[0], f1 = fac[fstep], f2 = fac[2 * fstep], f3 = fac[3 * fstep];
+          acc.x = fmaf(v0.x, f0, acc.x); acc.y = fmaf(v0.y, f0, acc.y); acc.z = fmaf(v0.z, f0, acc.z); acc.w = fmaf(v0.w, f0, acc.w);
+          acc.x = fmaf(v1.x, f1, acc.x); acc.y = fmaf(v1.y, f1, acc.y); acc.z = fmaf(v1.z, f1, acc.z); acc.w = fmaf(v1.w, f1, acc.w);
+          acc.x = fmaf(v2.x, f2, acc.x); acc.y = fmaf(v2.y, f2, acc.y); acc.z = fmaf(v2.z, f2, acc.z); acc.w = fmaf(v2.w, f2, acc.w);
+          acc.x = fmaf(v3.x, f3, acc.x); acc.y = fmaf(v3.y, f3, acc.y); acc.z = fmaf(v3.z, f3, acc.z); acc.w = fmaf(v3.w, f3, acc.w);
+        }
+        for (; n > 0; --n, p += step, fac += fstep) {
+          const float4 v0 = *reinterpret_cast<const float4*>(p);
+          const float f0 = fac[0];
+          acc.x = fmaf(v0.x, f0, acc.x); acc.y = fmaf(v0.y, f0, acc.y); acc.z = fmaf(v0.z, f0, acc.z); acc.w = fmaf(v0.w, f0, acc.w);
+        }
+      } else {
+        const float* p = sp + (size_t)iw * row_stride + (size_t)ih * kD + 4 * lane;
+        for (; n > 0; n -= 8) {
+          float4 v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          v[u] = s + u < splits ? __ldcg(reinterpret_cast<const float4*>(sp + ((size_t)(s + u) * g + h) * PS + c))
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int u = 0; u < 8; ++u)
+            v[u] = u < n ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)u * step)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const float f = s + u < splits ? cm[(s + u) * g + h] : 0.f;
-          acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
-          acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+          for (int u = 0; u < 8; ++u) {
+            const float f = u < n ? fac[u * fstep] : 0.f;
+            acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
+            acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+          }
+          p += 8 * step;
+          fac += 8 * fstep;
         }
       }
+      if (iw > 0) red[((size_t)(iw - 1) * g + ih) * 32 + lane] = acc;
     }
+    accs[k] = acc;
+  }
+  if (!landed && lane == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
+  if (ways > 1) __syncthreads();
+#pragma unroll
+  for (int k = 0; k < kHeadsPer; ++k) {
+    const int h = warp + k * kWarps;
+    if (h >= g) break;
+    float4 acc = accs[k];
+    for (int w = 1; w < ways; ++w) {
+      const float4 r = red[((size_t)(w - 1) * g + h) * 32 + lane];
+      acc.x += r.x; acc.y += r.y; acc.z += r.z; acc.w += r.w;
+    }
+    const int c = 4 * lane;
     if (ap.k_new) {
       const float fN = cN[h];
-      const uint2 vn = i == tid ? vn_pre : *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + c);
-      const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vn.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vn.y);
+      const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.y);
       acc.x = fmaf(__bfloat162float(v01.x), fN, acc.x); acc.y = fmaf(__bfloat162float(v01.y), fN, acc.y);
       acc.z = fmaf(__bfloat162float(v23.x), fN, acc.z); acc.w = fmaf(__bfloat162float(v23.y), fN, acc.w);
     }
+    const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
     if (raw_acc) {
-      const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
       *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = acc;
       if (c == 0) { raw_ml[2 * qh] = cM[h]; raw_ml[2 * qh + 1] = cL[h]; }
-      continue;
+    } else {
+      const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
+      __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + qh * kD + c);
+      o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+      o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
     }
-    const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
-    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + c);
-    o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-    o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
   }
   if (tid == 0 && !single) tickets[sl] = 0;   // ready for the next launch
 }
@@ -533,11 +744,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (kStages + 1) * sizeof(uint64_t);
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (kBars + kChunks) * sizeof(uint64_t);
 
 }  // namespace
 
 bool decode_mma_supported(const Geom& G) { return G.is_bf16 && G.d == kD && G.g <= 8; }
+int decode_mma_ctas_per_sm() { return kCtasPerSm; }
 
 // Tensor maps over the K and V arenas viewed as [total_rows, 128] bf16, boxes of 64 dims x 64 rows.
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out) {
@@ -572,10 +784,10 @@ void decode_mma_release(void* maps) { delete static_cast<DecodeMaps*>(maps); }
 
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st);
 
-// Scratch layout of all launches (as for launch_decode): ticket counters, then (stream, split, head)
-// partial rows.
+// Scratch layout of all launches: ticket counters, then (stream, split, head) rows of kD column sums,
+// then their (max, sum) pairs.
 // Un-normalised parts (see StepAppend::raw_acc) of the layer's streams, for decode merged over slots.
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
                                     float* scratch, int splits, int* status, const void* maps, int keys_only,
@@ -586,7 +798,7 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u};
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u, 0};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
                                                         tickets, status, ap, tm->k, tm->v);
   return cudaGetLastError();
@@ -604,7 +816,7 @@ cudaError_t launch_decode_parts_mma_slots(const Geom& G, const Arena& A, const i
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits, n_slots);
-  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words};
+  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words, 0};
   for (int i = 0; i < n_slots; ++i) ap.slot_layer[i] = slot_layers[i];
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, slot_layers[0], static_cast<const __nv_bfloat16*>(q), nullptr,
                                                         part, tickets, status, ap, tm->k, tm->v);
@@ -649,7 +861,7 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
 // [B*H, d] bf16; all streams of the layer have the same level-0 fill).  k_new == nullptr: plain decode.
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, cudaStream_t st) {
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st) {
   if (!maps) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
@@ -657,10 +869,11 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
   StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u};
+                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u, 0};
   if (seg_hint) {
     ap.n_seg = G.T + 1;
     for (int l = 0; l <= G.T; ++l) ap.seg[l] = seg_hint[l];
+    ap.early = early ? 1 : 0;
   }
   // programmatic stream serialization: back-to-back decode steps overlap a launch with the
   // previous kernel's tail (see the kernel's prologue)
