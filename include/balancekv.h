@@ -76,10 +76,22 @@ typedef struct balancekv_stats_t {
   int64_t device_status;      /* 0, or the first device-side error code                       */
   int64_t bytes_resident;     /* device memory owned by the context                           */
   int64_t kernels_launched;   /* kernels of this library launched so far                      */
+  int64_t walk_kernel;        /* Algorithm 2's kernel: 0 none (T = 0), 1 CUDA cores (fp32 FMA),
+                                 2 tensor cores (tcgen05); fixed at create time by the shape    */
+  int64_t decode_kernel;      /* decode attention: 1 CUDA cores, 2 tensor cores (mma + TMA)    */
 } balancekv_stats_t;
 
 /* Allocate a context: all cache memory for n_seqs*n_layers*n_kv_heads streams.
- * E_INVAL on a bad field, E_NOMEM / E_CUDA if the device allocation fails. */
+ * E_INVAL on a bad field, E_NOMEM / E_CUDA if the device allocation fails.  The kernels that
+ * serve the context follow from its shape (balancekv_stats reports them); if the tensor-core
+ * kernels of a shape that has them cannot be prepared, the call fails with E_CUDA -- there is no
+ * quiet change to other kernels.
+ *
+ * Device-side waits are bounded (about 50 ms).  One that gives up sets the context's status word:
+ * balancekv_stats then returns BALANCEKV_E_TIMEOUT (after filling the record), and so does every
+ * later call that would enqueue work once the host has seen the word (it is copied back behind
+ * every compress batch); results computed after that point are not valid.  balancekv_reset clears
+ * the condition. */
 int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out);
 int balancekv_destroy(balancekv_ctx* ctx);
 
@@ -151,20 +163,31 @@ int balancekv_decode_attn_host(balancekv_ctx* ctx, int layer, const void* q_host
  *
  * The split-K scratch is a fixed 8 MiB array inside the library image (held by every GPU
  * that loads the library, until the process exits); the call performs no cudaMalloc, cudaFree
- * or other allocating call.  A problem whose scratch (about n_streams * splits * group *
- * (head_dim+2) * 4 bytes, splits <= 64) exceeds the array is rejected with BALANCEKV_E_NOMEM
- * and a message on stderr.  The first call on a device looks up the array's device address
- * (cudaGetSymbolAddress); make that first call outside any stream capture.  All calls share
- * the array: the part a call uses is re-initialised by the call itself, but two calls that
- * overlap on the GPU (different CUDA streams) race on it -- issue them on one stream. */
+ * or other allocating call.  A problem whose scratch (256 bytes, a segment table of
+ * n_streams * (level+1) * 8 bytes, n_streams ticket words rounded up to 64, and n_streams *
+ * splits * group * (head_dim+4) * 4 bytes of partial rows, splits <= 64 chosen from the SM
+ * count) exceeds the array is rejected with BALANCEKV_E_NOMEM and a message on stderr.  The
+ * first call on a device -- of this function or of balancekv_decode_attn_static_status,
+ * whichever host thread gets there first -- looks up the array's device address
+ * (cudaGetSymbolAddress) and clears its status word with a synchronous memset; make that first
+ * call outside any stream capture.  All calls share the array: the part a call uses is
+ * re-initialised by the call itself, but two calls that overlap on the GPU (different CUDA
+ * streams) race on it -- issue them on one stream. */
 int balancekv_decode_attn_static(const void* K, const void* V, int n_streams, int cache_len, int n_heavy,
                                  int level, const void* q, void* out, int group, int head_dim, int dtype,
                                  void* stream);
+/* The entry point above returns before its kernel has run, so a bounded device-side wait that
+ * gives up cannot show in its return value; it sets a status word in the built-in array
+ * instead, which this call copies to *status_host (0 = fine, 1 = a wait gave up since the last
+ * read; the outputs of that launch are then not valid) and clears.  Allocates nothing;
+ * synchronises `stream`.  The paper has no counterpart. */
+int balancekv_decode_attn_static_status(int* status_host, void* stream);
 
 /* Load an already-compressed set into level `level` of every stream of one layer
  * (weight 2^level, the weights of Theorem 3.3's estimator): K, V: [n_seqs, n_kv_heads,
  * n_tokens, head_dim]; orig_idx (may be NULL): [n_seqs, n_kv_heads, n_tokens] original
- * token positions.  level in [0, T]; for 1 <= level < T at most t rows fit. */
+ * token positions.  level is 0 or T (else BALANCEKV_E_INVAL): the levels between hold exactly 0
+ * or t/2 rows by construction and are only ever filled by balancekv_compress. */
 int balancekv_cache_load_level(balancekv_ctx* ctx, int layer, int level, const void* K, const void* V,
                                const int32_t* orig_idx, int n_tokens, void* stream);
 
@@ -270,6 +293,11 @@ int balancekv_profile_enable(balancekv_ctx* ctx, int on);
 int balancekv_profile_sample(balancekv_ctx* ctx, int kernel_class, int every);
 int balancekv_profile_read(balancekv_ctx* ctx, double* out_host);
 
+/* Testing aid: overwrite the context's device status word (0 = clear, 1 = a wait gave up), as a
+ * kernel whose bounded wait ran out would.  Synchronises the device. */
+int balancekv_debug_set_status(balancekv_ctx* ctx, int value);
+
+/* Synchronises the device.  Returns BALANCEKV_E_TIMEOUT (record filled) if a device-side wait gave up. */
 int balancekv_stats(balancekv_ctx* ctx, balancekv_stats_t* out);
 const char* balancekv_strerror(int code);
 

@@ -6,6 +6,7 @@ from .binding import (  # noqa: E402,F401
     EXPORTS,
     LIB_PATH,
     decode_attn_static,
+    decode_attn_static_status,
     load,
     plan_calls,
 )

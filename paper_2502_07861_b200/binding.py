@@ -24,7 +24,7 @@ EXPORTS = [
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
     "balancekv_decode_attn_two", "balancekv_decode_attn_merged", "balancekv_stream_append_bucketed",
-    "balancekv_stream_append_layer_bucketed",
+    "balancekv_stream_append_layer_bucketed", "balancekv_debug_set_status", "balancekv_decode_attn_static_status",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -51,7 +51,8 @@ class Config(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("tokens_appended", "tokens_stored", "calls_run", "walk_fails",
-                                         "device_status", "bytes_resident", "kernels_launched")]
+                                         "device_status", "bytes_resident", "kernels_launched", "walk_kernel",
+                                         "decode_kernel")]
 
 
 def load():
@@ -95,6 +96,8 @@ def load():
     lib.balancekv_stream_append_bucketed.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
     lib.balancekv_stream_append_layer_bucketed.argtypes = [vp, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
+    lib.balancekv_decode_attn_static_status.argtypes = [vp, vp]
+    lib.balancekv_debug_set_status.argtypes = [vp, ci]
     for name in EXPORTS:
         if name != "balancekv_strerror":
             getattr(lib, name).restype = ci
@@ -342,6 +345,10 @@ class Context:
         return (_from_ptr(pe.value, (m.value,), torch.int8), _from_ptr(ps.value, (m.value,), torch.float32),
                 _from_ptr(pp.value, (m.value,), torch.float32))
 
+    def debug_set_status(self, value):
+        """Testing aid: overwrite the device status word (1 = a bounded wait gave up)."""
+        _check(self.lib.balancekv_debug_set_status(self._h, int(value)), "balancekv_debug_set_status")
+
     def reset(self, stream=None):
         _check(self.lib.balancekv_reset(self._h, _stream_ptr(stream)), "balancekv_reset")
 
@@ -365,7 +372,9 @@ class Context:
 
     def stats(self):
         s = Stats()
-        _check(self.lib.balancekv_stats(self._h, C.byref(s)), "balancekv_stats")
+        code = self.lib.balancekv_stats(self._h, C.byref(s))
+        if code != E_TIMEOUT:               # a timed-out wait is reported through device_status; the record is filled
+            _check(code, "balancekv_stats")
         return {n: getattr(s, n) for n, _ in Stats._fields_}
 
 
@@ -387,6 +396,14 @@ def decode_attn_static(K, V, n_heavy, level, q, out=None, stream=None):
                                                C.c_void_p(out.data_ptr()), q.shape[1], K.shape[2], dtype_code,
                                                _stream_ptr(stream)), "balancekv_decode_attn_static")
     return out
+
+
+def decode_attn_static_status(stream=None):
+    """Status word of the allocation-free entry point on the current device: 0, or 1 if a bounded
+    wait of one of its launches gave up since the last read (reading clears it).  Synchronises the stream."""
+    v = C.c_int(0)
+    _check(load().balancekv_decode_attn_static_status(C.byref(v), _stream_ptr(stream)), "balancekv_decode_attn_static_status")
+    return v.value
 
 
 class _RawDevice:

@@ -66,6 +66,7 @@ struct balancekv_ctx {
   int8_t* d_eta = nullptr;
   unsigned long long* d_fail = nullptr;
   int* d_status = nullptr;
+  int* h_status = nullptr;       // pinned mirror of the status word, refreshed after every compress batch and by stats
   float* d_decode_scratch = nullptr;
   int max_splits = 1;
   int decode_slots = 148;        // CTAs of the decode kernel that are resident at once
@@ -211,6 +212,10 @@ int64_t dbg_offset(const balancekv_ctx* c, int stream, int level, int64_t ordina
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// A bounded device-side wait that gave up sets the context's status word.  The host sees it through
+// a pinned mirror (no synchronisation): once set, every call that would enqueue more work refuses.
+bool timed_out(const balancekv_ctx* c) { return c->h_status && *static_cast<volatile int*>(c->h_status) == kStatusWaitTimeout; }
+
 int check_config(const balancekv_config& f) {
   if (f.n_seqs < 1 || f.n_layers < 1 || f.n_kv_heads < 1 || f.n_q_heads < 1) return BALANCEKV_E_INVAL;
   if (f.n_layers > 65535 || f.n_kv_heads > 65535) return BALANCEKV_E_INVAL;
@@ -337,6 +342,8 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   if ((rc = dev_alloc(c, &c->d_fail, 1))) return fail(rc);
   if ((rc = dev_alloc(c, &c->d_status, 1))) return fail(rc);
   if (cudaMemset(c->d_fail, 0, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+  if (cudaMallocHost(reinterpret_cast<void**>(&c->h_status), 64) != cudaSuccess) return fail(BALANCEKV_E_NOMEM);
+  *c->h_status = 0;
   {
     const int n_sl = f.n_seqs * f.n_kv_heads;
     const int per_sm = f.gram_path != 1 && decode_mma_supported(G) ? decode_mma_ctas_per_sm() : 2;
@@ -353,18 +360,16 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   for (int i = 0; i < 2; ++i)
     if (cudaEventCreateWithFlags(&c->ring_ev[i], cudaEventDisableTiming) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
 
-  if (f.gram_path != 1 && decode_mma_supported(G)) {
-    if (decode_mma_prepare(G, c->A, c->total_rows, &c->decode_maps) != cudaSuccess) c->decode_maps = nullptr;
+  // The kernel family follows from the shape alone; a supported shape whose tensor maps cannot be
+  // prepared is an error, never a quiet change of kernels.
+  const bool rows_ok = c->total_rows < ((int64_t)1 << 31);
+  if (f.gram_path != 1 && decode_mma_supported(G) && rows_ok) {
+    if (decode_mma_prepare(G, c->A, c->total_rows, &c->decode_maps) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   }
-  const bool tc_ok = walk_tc_supported(G) && c->total_rows < ((int64_t)1 << 31);
+  const bool tc_ok = walk_tc_supported(G) && rows_ok;
   if (f.gram_path == 2 && !tc_ok) return fail(BALANCEKV_E_INVAL);
   c->use_tc = T > 0 && tc_ok && f.gram_path != 1;
-  if (c->use_tc) {
-    if (walk_tc_prepare(G, c->A, c->total_rows, &c->tmaps) != cudaSuccess) {
-      if (f.gram_path == 2) return fail(BALANCEKV_E_CUDA);
-      c->use_tc = false;
-    }
-  }
+  if (c->use_tc && walk_tc_prepare(G, c->A, c->total_rows, &c->tmaps) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   if (T > 0 && !c->use_tc) {
     if (!walk_simt_supported(G.d)) return fail(BALANCEKV_E_INVAL);
     if (walk_simt_smem_bytes(G.d, t) > (size_t)227 * 1024) return fail(BALANCEKV_E_INVAL);
@@ -388,6 +393,7 @@ int balancekv_destroy(balancekv_ctx* c) {
     if (p) cudaFree(p);
   if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
   if (c->h_ring) cudaFreeHost(c->h_ring);
+  if (c->h_status) cudaFreeHost(c->h_status);
   if (c->step_host) cudaFreeHost(c->step_host);
   if (c->step_copy_stream) cudaStreamDestroy(c->step_copy_stream);
   for (cudaEvent_t e : c->step_used_ev)
@@ -408,6 +414,7 @@ static int append_impl(balancekv_ctx* c, const std::vector<int>& streams, int le
   if (!K || !V || n < 0) return BALANCEKV_E_INVAL;
   if (!aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
   if (n == 0) return BALANCEKV_OK;
+  if (timed_out(c)) return BALANCEKV_E_TIMEOUT;
   c->decode_chain = false;
   const balancekv_config& f = c->cfg;
   const Layout& Lo = c->Lo;
@@ -621,11 +628,14 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
     BKV_CUDA(launch_seg_update(c->A, static_cast<const SegUpdate*>(d_segs), (int)P.segs.size(), st));
     c->kernels_launched++;
   }
+  // refresh the host's view of the status word behind the batch (4 bytes, no synchronisation)
+  BKV_CUDA(cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
   return BALANCEKV_OK;
 }
 
 static int compress_streams(balancekv_ctx* c, const std::vector<int>& streams, int T, cudaStream_t st) {
   if (T != c->cfg.levels) return BALANCEKV_E_INVAL;
+  if (timed_out(c)) return BALANCEKV_E_TIMEOUT;
   for (int s : streams) c->st[s].pending = 0;
   if (T == 0) return BALANCEKV_OK;
   // greedy batches of at most max_calls level-0 calls
@@ -706,6 +716,7 @@ static int pick_splits(balancekv_ctx* c, int layer) {
 int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || !q || !out) return BALANCEKV_E_INVAL;
   if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
+  if (timed_out(c)) return BALANCEKV_E_TIMEOUT;
   const int splits = pick_splits(c, layer);
   {
     ProfScope ps(c, 4, static_cast<cudaStream_t>(stream));
@@ -772,6 +783,7 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
   if (!c || !q || !out || !layers_num || !layers_den || n_num < 1 || n_den < 1) return BALANCEKV_E_INVAL;
   if (!aligned16(q) || !aligned16(out)) return BALANCEKV_E_INVAL;
   if (!c->decode_maps) return BALANCEKV_E_INVAL;          // bf16, head_dim 128, group <= 8 only
+  if (timed_out(c)) return BALANCEKV_E_TIMEOUT;
   c->decode_chain = false;
   // distinct slots in order of first appearance, with the sides they enter
   int slots[BALANCEKV_MAX_MERGE];
@@ -832,6 +844,7 @@ int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, co
 
 int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                           void* stream) {
+  if (c && timed_out(c)) return BALANCEKV_E_TIMEOUT;
   // One launch when the tensor-core decode kernel serves this context and the layer's streams are
   // in lockstep with room for the token: the kernel appends after attending (see its header).
   if (c && layer >= 0 && layer < c->cfg.n_layers && c->decode_maps && q && out && k_new && v_new && aligned16(q) &&
@@ -1028,6 +1041,7 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
   if (i_top < -60 || i_top > 60 || !(rho >= 0.f) || rho > 1.f) return BALANCEKV_E_INVAL;
   const int n_sl = (int)heads.size();
   if (n_sl < 1) return BALANCEKV_E_INVAL;
+  if (timed_out(c)) return BALANCEKV_E_TIMEOUT;
   c->decode_chain = false;
   if (c->bucket_vmax2.empty()) {
     c->bucket_vmax2.assign(c->n_streams, 0.f);
@@ -1160,6 +1174,9 @@ int balancekv_reset(balancekv_ctx* c, void* stream) {
   c->bucket_vmax2.clear();
   c->bucket_erase_max.clear();
   BKV_CUDA(cudaMemsetAsync(c->A.seg, 0, sizeof(Seg) * (size_t)c->n_streams * (c->cfg.levels + 1), st));
+  // a context that gave up on a device-side wait becomes usable again
+  BKV_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(int), st));
+  *c->h_status = 0;
   return BALANCEKV_OK;
 }
 
@@ -1214,6 +1231,17 @@ int balancekv_stats(balancekv_ctx* c, balancekv_stats_t* out) {
   out->device_status = status;
   out->bytes_resident = (int64_t)c->bytes_resident;
   out->kernels_launched = c->kernels_launched;
+  out->walk_kernel = c->cfg.levels == 0 ? 0 : (c->use_tc ? 2 : 1);
+  out->decode_kernel = c->decode_maps ? 2 : 1;
+  if (c->h_status) *c->h_status = status;
+  return status == kStatusWaitTimeout ? BALANCEKV_E_TIMEOUT : BALANCEKV_OK;
+}
+
+int balancekv_debug_set_status(balancekv_ctx* c, int value) {
+  if (!c) return BALANCEKV_E_INVAL;
+  BKV_CUDA(cudaDeviceSynchronize());
+  BKV_CUDA(cudaMemcpy(c->d_status, &value, sizeof(int), cudaMemcpyHostToDevice));
+  *c->h_status = value;
   return BALANCEKV_OK;
 }
 

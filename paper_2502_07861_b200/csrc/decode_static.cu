@@ -13,6 +13,7 @@
 // kStaticBytes until the process exits.  In host code the array's name is only a handle; the
 // device address is obtained once per device with cudaGetSymbolAddress.
 #include <cstdio>
+#include <mutex>
 
 #include "../../include/balancekv.h"
 #include "common.cuh"
@@ -27,12 +28,14 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices] = {};    // device address of the array, per device
 int g_sm_count[kMaxDevices] = {};
+std::once_flag g_setup_once[kMaxDevices];           // the per-device set-up runs once, whichever host thread comes first
+cudaError_t g_setup_err[kMaxDevices] = {};
 
-// Layout inside the array: [status word, 256 B][segment table][tickets + partials].
+// Layout inside the array: [status word, 256 B][segment table][tickets + partials].  The status word
+// is left alone here: it keeps the first failure until balancekv_decode_attn_static_status reads it.
 __global__ void static_setup_kernel(unsigned char* base, int n_streams, int T, int n_heavy, int n_tail,
                                     size_t seg_off, size_t scratch_off) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i == 0) *reinterpret_cast<int*>(base) = 0;
   if (i < n_streams) {
     Seg* seg = reinterpret_cast<Seg*>(base + seg_off) + (size_t)i * (T + 1);
     for (int l = 0; l <= T; ++l) seg[l] = Seg{0, 0};
@@ -41,6 +44,38 @@ __global__ void static_setup_kernel(unsigned char* base, int n_streams, int T, i
     else seg[0] = Seg{0, n_heavy + n_tail};
     reinterpret_cast<unsigned*>(base + scratch_off)[i] = 0u;   // ticket counter of the stream
   }
+}
+
+// Once per device, with that device current: resolve the array's device address (in host code the
+// array's name is only a handle) and clear the status word.  The array is not otherwise initialised:
+// every call sets up the part it uses.
+void static_setup_device(int dev) {
+  void* p = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+  if (e == cudaSuccess && !p) e = cudaErrorInvalidSymbol;
+  int sms = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess && sms < 1) e = cudaErrorInvalidValue;
+  if (e == cudaSuccess) e = cudaMemset(p, 0, 256);
+  g_setup_err[dev] = e;
+  if (e != cudaSuccess) return;
+  g_sm_count[dev] = sms;
+  g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+}
+
+// 0 on success, with the current device's index in *dev_out.
+int static_device(int* dev_out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return BALANCEKV_E_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return BALANCEKV_E_INVAL;
+  std::call_once(g_setup_once[dev], static_setup_device, dev);
+  if (g_setup_err[dev] != cudaSuccess || !g_scratch_addr[dev]) {
+    std::fprintf(stderr, "balancekv_decode_attn_static: set-up of the built-in scratch array failed: %s\n",
+                 cudaGetErrorString(g_setup_err[dev]));
+    return BALANCEKV_E_CUDA;
+  }
+  *dev_out = dev;
+  return BALANCEKV_OK;
 }
 
 }  // namespace
@@ -60,21 +95,7 @@ extern "C" int balancekv_decode_attn_static(const void* K, const void* V, int n_
                           reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out);
   if (align & 15) return BALANCEKV_E_INVAL;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return BALANCEKV_E_CUDA;
-  if (dev < 0 || dev >= kMaxDevices) return BALANCEKV_E_INVAL;
-  if (!g_scratch_addr[dev]) {
-    // once per device, with that device current: resolve the array's device address
-    void* p = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
-    if (e != cudaSuccess || !p) {
-      std::fprintf(stderr, "balancekv_decode_attn_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
-      return BALANCEKV_E_CUDA;
-    }
-    int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return BALANCEKV_E_CUDA;
-    g_sm_count[dev] = sms;
-    g_scratch_addr[dev] = static_cast<unsigned char*>(p);
-  }
+  if (int rc = static_device(&dev)) return rc;
   unsigned char* base = g_scratch_addr[dev];
   const int esz = dtype ? 2 : 4;
   const int T = level;
@@ -117,5 +138,19 @@ extern "C" int balancekv_decode_attn_static(const void* K, const void* V, int n_
     std::fprintf(stderr, "balancekv_decode_attn_static: launch failed: %s\n", cudaGetErrorString(e));
     return BALANCEKV_E_CUDA;
   }
+  return BALANCEKV_OK;
+}
+
+extern "C" int balancekv_decode_attn_static_status(int* status_host, void* stream) {
+  if (!status_host) return BALANCEKV_E_INVAL;
+  int dev = 0;
+  if (int rc = static_device(&dev)) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int v = 0;
+  // read, then clear, in stream order behind the launches issued so far on `stream`
+  if (cudaMemcpyAsync(&v, g_scratch_addr[dev], sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return BALANCEKV_E_CUDA;
+  if (cudaMemsetAsync(g_scratch_addr[dev], 0, sizeof(int), st) != cudaSuccess) return BALANCEKV_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BALANCEKV_E_CUDA;
+  *status_host = v;
   return BALANCEKV_OK;
 }

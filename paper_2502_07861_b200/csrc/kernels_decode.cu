@@ -23,7 +23,8 @@ constexpr int kThreads = 256;
 constexpr int kWarps = 8;
 constexpr int kStages = 3;
 constexpr int kTileBytes = 16384;          // per tensor per stage
-constexpr long long kWaitCycles = 4000000000LL;
+constexpr int kMaxDevices = 64;
+constexpr long long kWaitCycles = 100000000LL;    // about 50 ms: a bulk copy that has not landed by then never will
 
 __device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -323,11 +324,15 @@ cudaError_t launch_t(const Geom& G, const Arena& A, int layer, const void* q, vo
                      int splits, int* status, cudaStream_t st) {
   auto kern = decode_kernel<kBf16, D, GQ>;
   const size_t smem = (size_t)kStages * 2 * kTileBytes + kStages * sizeof(uint64_t);
-  static bool configured = false;   // one device per process uses this library
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // the attribute belongs to the (kernel, device) pair: once per device that launches this instance
+  static bool configured[kMaxDevices] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
   }
   const int n_sl = G.B * G.H;
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);

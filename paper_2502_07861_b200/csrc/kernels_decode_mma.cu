@@ -47,7 +47,7 @@ constexpr int kD = 128;
 constexpr uint32_t kHalf = kTN * 128;        // bytes of one [64 tokens][64 dims] bf16 box
 constexpr uint32_t kTensorBytes = 2 * kHalf; // K (or V) tile: two boxes
 constexpr uint32_t kStageBytes = 2 * kTensorBytes;
-constexpr long long kWaitCycles = 200000000LL;   // about 0.1 s: a bulk copy that has not landed by then never will
+constexpr long long kWaitCycles = 100000000LL;   // about 50 ms: a bulk copy that has not landed by then never will
 constexpr int kChunks = 1;                   // barriers of the combine's staging copy
 constexpr int PS = kD + 4;                   // row of the in-CTA merge buffer: acc[D], max, sum, 2 pad (bank-conflict free)
 

@@ -45,7 +45,7 @@ constexpr int kThreads = 32 * (kEpiWarps + 3);
 constexpr uint32_t kHalfBytes = 16384;     // [128 rows][64 bf16] = one swizzle-atom column of a tile
 constexpr uint32_t kTileBytes = 32768;     // [128 rows][128 bf16]
 constexpr uint32_t kTmemCols = 512;
-constexpr long long kWaitCycles = 4000000000LL;
+constexpr long long kWaitCycles = 100000000LL;   // about 50 ms; every wait here is on this CTA's own copies and MMAs
 
 struct TensorMaps {
   CUtensorMap k, v;

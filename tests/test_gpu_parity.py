@@ -262,3 +262,30 @@ def test_degenerate_inputs_zero_values_and_duplicate_tokens(cuda_lib, gram):
             assert np.all(hz.ctx.decode_attn(0, to_device(q, "bf16")).float().cpu().numpy() == 0)
         else:
             hz.check_decode(l, q, DEC_TOL["bf16"])
+
+
+def test_a_timed_out_wait_surfaces_as_an_error_code_and_reset_clears_it(cuda_lib):
+    """A bounded device-side wait that gives up sets the context's status word; here the word is set
+    from the host (no kernel is made to hang).  stats() then reports it, every call that would
+    enqueue work is refused with BALANCEKV_E_TIMEOUT, and reset() makes the context usable again."""
+    bk = cuda_lib
+    ctx = bk.Context(n_seqs=1, n_layers=1, n_kv_heads=2, n_q_heads=8, head_dim=128, dtype="bf16", block=128, levels=1,
+                     max_tokens=1024)
+    K = torch.randn(1, 2, 256, 128, device="cuda").to(torch.bfloat16)
+    q = torch.randn(1, 8, 128, device="cuda").to(torch.bfloat16)
+    ctx.stream_append_layer(0, K, K)
+    ctx.compress()
+    st = ctx.stats()
+    assert st["device_status"] == 0 and st["walk_kernel"] == 2 and st["decode_kernel"] == 2
+    ctx.debug_set_status(1)
+    assert ctx.stats()["device_status"] == 1
+    for call in (lambda: ctx.decode_attn(0, q), lambda: ctx.stream_append_layer(0, K, K), lambda: ctx.compress()):
+        with pytest.raises(bk.BalanceKVError) as ei:
+            call()
+        assert ei.value.code == bk.binding.E_TIMEOUT
+    ctx.reset()
+    ctx.stream_append_layer(0, K, K)
+    ctx.compress()
+    ctx.decode_attn(0, q)
+    assert ctx.stats()["device_status"] == 0
+    ctx.close()

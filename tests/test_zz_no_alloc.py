@@ -2,9 +2,10 @@
 
 balancekv_decode_attn_static serves callers that may not allocate device memory (latency
 critical loops, plugins fed with framework-owned buffers, fully committed memory pools): its
-scratch is a fixed array inside the library.  Here it must reproduce balancekv_decode_attn,
-within the decode tolerance of the other GPU tests, on two calls in a row (the second call
-reuses the array the first one left behind).  This file sorts last on purpose."""
+scratch is a fixed array inside the library.  Here it must reproduce balancekv_decode_attn
+and the CPU oracle's weighted attention, within the decode tolerance of the other GPU tests, on
+two calls in a row (the second call reuses the array the first one left behind), without taking
+any device memory and without tripping a bounded wait.  This file sorts last on purpose."""
 import numpy as np
 import pytest
 import torch
@@ -35,15 +36,32 @@ def test_static_scratch_decode_matches_context_decode_twice(cuda_lib, dtype, d, 
         ctx.stream_append_layer(0, Kd[:, :, n_heavy:].contiguous(), Vd[:, :, n_heavy:].contiguous())
     Ks, Vs = Kd.reshape(B * H, n, d), Vd.reshape(B * H, n, d)
     out_static = torch.empty(B * H, g, d, dtype=Kd.dtype, device="cuda")
+    import oracle
+
+    w = np.concatenate([np.full(n_heavy, float(1 << T)), np.ones(n_tail)])
     for call in range(2):                                   # two calls in a row share the built-in array
-        q = _dev(synth.queries(90, 0, call, B, H * g, d, dtype), dtype)
+        qh = synth.queries(90, 0, call, B, H * g, d, dtype)
+        q = _dev(qh, dtype)
         ref = ctx.decode_attn(0, q).float().cpu().numpy().reshape(B * H, g, d)
         out_static.fill_(float("nan"))
-        bk.decode_attn_static(Ks, Vs, n_heavy, T, q.reshape(B * H, g, d), out_static)
+        qs = q.reshape(B * H, g, d)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]          # device-wide free memory, not torch's pool
+        bk.decode_attn_static(Ks, Vs, n_heavy, T, qs, out_static)
+        torch.cuda.synchronize()
+        if call == 1:                                       # the first call on a device may load the kernel image
+            assert torch.cuda.mem_get_info()[0] == free_before, "the allocation-free entry point took device memory"
         got = out_static.float().cpu().numpy()
         assert np.isfinite(got).all()
         err = np.linalg.norm(got - ref) / np.linalg.norm(ref)
         assert err <= DEC_TOL[dtype], (call, err)
+        # the definition itself: Theorem 3.3's estimator over the caller's rows, by the CPU oracle
+        for s in range(B * H):
+            exact = oracle.weighted_attention(K.reshape(B * H, n, d)[s], V.reshape(B * H, n, d)[s], w,
+                                              qh.reshape(B * H, g, d)[s])
+            e2 = np.linalg.norm(got[s] - exact) / np.linalg.norm(exact)
+            assert e2 <= DEC_TOL[dtype], (call, s, e2)
+        assert bk.decode_attn_static_status() == 0          # no bounded wait gave up
     ctx.close()
 
 
