@@ -133,27 +133,133 @@ def oracle_sample(w, K, V, q, sample_tokens, decode_steps):
 
 
 def run_reference(args, w):
-    """CPU oracle arm: each step is a bounded sample (1/8 of the context per stream)."""
+    """CPU oracle arm on the product arm's workload: every step is the whole context of every stream
+    and all decode steps.  The oracle needs several seconds per step, so at most as many of the
+    requested steps run as fit in about three minutes (the line says how many)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample, dsteps = w["context"] // 8, w["decode_steps"] // 8
     K, V, q = make_inputs(w, w["context"], w["decode_steps"])
     for _ in range(min(args.warmup, 1)):
         oracle_sample(w, K, V, q, w["block"] * 2, 1)
-    times = []
-    for _ in range(args.steps):
-        dt, units, threads, _ = oracle_sample(w, K, V, q, sample, dsteps)
+    times, budget_s = [], 180.0
+    units = threads = 0
+    for i in range(args.steps):
+        dt, units, threads, _ = oracle_sample(w, K, V, q, w["context"], w["decode_steps"])
         times.append(dt)
+        if sum(times) + dt > budget_s:
+            break
     val = units * len(times) / sum(times)
-    sample_txt = f"first {sample} of {w['context']} context tokens of each of the {w['n_kv_heads']} streams + {dsteps} decode steps"
-    line = dict(metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
-                ms_per_step=1e3 * float(np.mean(times)), higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype="f64", data="synthetic", impl="reference",
-                config=dict(workload=w["name"], sample=sample_txt, context=w["context"], block=w["block"], levels=w["levels"]),
+    sample_txt = (f"all {w['context']} context tokens of each of the {w['n_kv_heads']} streams + all {w['decode_steps']} decode "
+                  f"steps per step; {len(times)} of the {args.steps} requested steps run (time budget {budget_s:.0f} s)")
+    line = dict(metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=len(times), steps_requested=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * float(np.mean(times)), higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=w["name"], n_kv_heads=w["n_kv_heads"], n_q_heads=w["n_q_heads"], head_dim=w["head_dim"],
+                            context=w["context"], block=w["block"], levels=w["levels"], decode_steps=w["decode_steps"]),
                 cpu_baseline=dict(value=val, unit=UNIT, cores=threads, kind="oracle", sample=sample_txt),
                 e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
+
+
+def source_digest(*names):
+    """sha256 over the named kernel sources: an ncu traffic figure is only quoted for the code it was taken from."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2502_07861_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(shape):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the graded kernels from the
+    ncu captures summarised under profiles/: entries of profiles/traffic.json that match this shape and
+    whose kernel source is unchanged since the capture; anything else is reported as null."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    out = {}
+    if not os.path.exists(path):
+        return out
+    for e in json.load(open(path)).get("entries", []):
+        if e.get("shape") == shape and e.get("source_digest") == source_digest(*e.get("sources", [])):
+            out[e["kernel"]] = float(e["dram_bytes_per_launch"])
+    return out
+
+
+def per_config(peaks):
+    """The other configurations as bounded slices (each a few hundred milliseconds of GPU time): what was
+    run, the figures, and how a slice relates to the whole configuration."""
+    import torch
+
+    import paper_2502_07861_b200 as bk
+    from paper_2502_07861_b200 import microbench, synth
+
+    out = {}
+    # config 1: the tiny fp32 stream (CUDA-core kernels), time only
+    n, t, d = 1024, 256, 64
+    Kf, Vf = synth.stream_kv("outlier2", 1001, 0, 0, 0, n, d, "fp32")
+    K = torch.from_numpy(Kf)[None, None].cuda().contiguous()
+    V = torch.from_numpy(Vf)[None, None].cuda().contiguous()
+    qs = torch.from_numpy(synth.queries(1001, 0, 0, 16, 1, d, "fp32")).cuda().contiguous()    # 16 queries
+    ctx = bk.Context(n_seqs=1, n_layers=1, n_kv_heads=1, n_q_heads=1, head_dim=d, dtype="fp32", block=t, levels=1, max_tokens=n)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    tc, td = [], []
+    for it in range(8):
+        ctx.reset()
+        ev[0].record()
+        for b in range(n // t):
+            ctx.stream_append_layer(0, K[:, :, b * t:(b + 1) * t].contiguous(), V[:, :, b * t:(b + 1) * t].contiguous())
+            ctx.compress()
+        ev[1].record()
+        for i in range(16):
+            ctx.decode_attn(0, qs[i:i + 1])
+        ev[2].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            tc.append(ev[0].elapsed_time(ev[1])); td.append(ev[1].elapsed_time(ev[2]))
+    st = ctx.stats()
+    ctx.close()
+    out["config1_tiny_fp32"] = dict(
+        workload="1 stream, d=64, fp32, 1024 tokens in blocks of 256, T=1, 16 decode queries", slice="whole configuration",
+        append_compress_us=1e3 * float(np.mean(tc)), decode_us_per_query=1e3 * float(np.mean(td)) / 16,
+        walk_kernel=int(st["walk_kernel"]), decode_kernel=int(st["decode_kernel"]),
+        note="launch-latency bound (4 calls of 256 tokens): time only, no roofline claim")
+    del K, V, ctx
+
+    def compress_entry(res, workload, slice_txt, rule):
+        return dict(workload=workload, slice=slice_txt, extrapolation=rule, compress_ms=res["compress_ms"],
+                    compress_token_heads_per_s=res["token_heads_per_s"], calls=res["calls"],
+                    gram_walk=dict(bound="tensor", achieved=res["gram_walk_tflops"], peak=peaks["tensor"], unit="TFLOP/s",
+                                   frac=res["gram_walk_tflops"] / peaks["tensor"], ms=res["gram_walk_ms"]),
+                    compact=dict(bound="hbm", achieved=res["compact_gbs"], peak=peaks["hbm"], unit="GB/s",
+                                 frac=res["compact_gbs"] / peaks["hbm"], ms=res["compact_ms"]),
+                    walk_kernel=res["walk_kernel"], device_status=res["device_status"])
+
+    # config 3: one 8192-token prefill chunk of all 4 x 32 x 8 streams (t = 2048, T = 2)
+    r3 = microbench.compress_case(4 * 32 * 8, 128, 8192, 2048, 2, iters=3)
+    out["config3_8b_stack"] = compress_entry(
+        r3, "4 sequences x 32 layers x 8 KV heads, d=128, bf16, t=2048, T=2",
+        "one 8192-token prefill chunk of all 1024 streams (1 of 16 chunks), compress only",
+        "whole configuration = 16 such chunks (work is linear in the context at fixed t); decode: see config5")
+    # config 4: one chunk of 16 of the 48 layers (8 x 16 x 8 streams), t = 1024, T = 3, recent window 128
+    r4 = microbench.compress_case(8 * 16 * 8, 128, 8192, 1024, 3, iters=3, window=128)
+    out["config4_14b"] = compress_entry(
+        r4, "8 sequences x 48 layers x 8 KV heads, d=128, bf16, t=1024, T=3, recent window 128",
+        "one 8192-token prefill chunk of 16 of the 48 layers (1024 of 3072 streams), compress only",
+        "whole configuration = 3 x 8 such slices (linear in streams and context)")
+    # config 5: decode sweep at the 32B shape; distinct layers are cycled so that no launch re-reads L2
+    sweep = []
+    for Lc in (2048, 4096, 8192, 16384, 32768):
+        r = microbench.decode_case(32, 8, 5, 128, Lc, 2, iters=30, max_layers=8)
+        sweep.append(dict(cache_len=Lc, us_per_layer=r["us_per_layer"], us_x64_layers=64 * r["us_per_layer"],
+                          achieved=r["achieved_gbs"], frac=r["frac"], layers_cycled=r["layers_cycled"],
+                          device_status=r["device_status"]))
+    out["config5_decode_sweep"] = dict(
+        workload="batch 32 x 8 KV heads x 5 query heads each, d=128, bf16, weights 2^2, cache loaded at level T",
+        slice="one layer per launch; 64 layers = 64 such launches", bound="hbm", peak=peaks["hbm"], unit="GB/s",
+        points=sweep)
+    return out
 
 
 def main():
@@ -164,6 +270,7 @@ def main():
     ap.add_argument("--impl", default="balancekv")
     ap.add_argument("--gram-path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the slices of the other configurations")
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling a small case)")
     ap.add_argument("--decode-steps", type=int, default=None)
     args = ap.parse_args()
@@ -308,10 +415,9 @@ def main():
     # time share of each kernel class in the timed region
     dc_launches = n_dec * args.steps
     dc_total_ms = dc_ms
-    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-    # summarised under profiles/ (average of the level-0 and level-1 launches; the decode figure is
-    # a cold-L2 launch of the same shape, while this loop re-reads its cache from L2)
-    traffic = dict(gram_walk=105.4e6, compact=67.5e6, decode=33.65e6) if (n_ctx, t, T, B * H) == (32768, 1024, 2, 8) else {}
+    # DRAM bytes per launch from the ncu captures summarised under profiles/ (see measured_traffic); the
+    # decode figure is a cold-L2 launch of the same shape, while this loop re-reads its cache from L2
+    traffic = measured_traffic(dict(context=n_ctx, block=t, levels=T, streams=B * H))
     kernels = dict(
         gram_walk=dict(bound="tensor", achieved=tensor_ach, peak=peaks["tensor"], unit="TFLOP/s",
                        frac=tensor_ach / peaks["tensor"], traffic=traffic.get("gram_walk"), ms_per_launch=gw_ms_per_launch, launches=gw_n,
@@ -337,12 +443,19 @@ def main():
         cpu = dict(value=units / scaled, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
                    sample=f"all {n_ctx} context tokens of each of the {B * H} streams + {dsteps} of the {n_dec} decode steps "
                           f"(their time scaled to {n_dec})")
+    pc = None
+    if not args.no_per_config and world == 1 and (n_ctx, n_dec) == (WORKLOAD["context"], WORKLOAD["decode_steps"]):
+        ctx.close()
+        del K_ctx, V_ctx, flush
+        torch.cuda.empty_cache()
+        pc = per_config(peaks)
     line = dict(
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
         data="synthetic",
         config=dict(workload=w["name"], n_kv_heads=H, n_q_heads=Hq, head_dim=d, context=n_ctx, block=t, levels=T,
-                    decode_steps=n_dec, gram_path="tcgen05" if False else ("auto" if args.gram_path == 0 else args.gram_path),
+                    decode_steps=n_dec, walk_kernel={0: "none", 1: "cuda-core fp32", 2: "tcgen05"}[int(status["walk_kernel"])],
+                    decode_kernel={1: "cuda-core", 2: "mma.sync + TMA"}[int(status["decode_kernel"])],
                     l2="flushed between steps (256 MB write, outside the event brackets); inputs 134 MB > L2",
                     replicas_per_gpu=1),
         compress_tokens_per_s=units_per_step / (float(t_comp.mean()) * 1e-3),
@@ -353,7 +466,7 @@ def main():
         e2e=dict(value=world * units_per_step * e2e_steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                  ms_per_step=1e3 * e2e_s / e2e_steps, timing="wall clock, synchronised on both sides"),
         gpu_launches=int(launches), clocks=clocks, cpu_baseline=cpu,
-        device_status=int(status["device_status"]), walk_fails=int(status["walk_fails"]),
+        device_status=int(status["device_status"]), walk_fails=int(status["walk_fails"]), per_config=pc,
     )
     print(json.dumps(line))
     if world > 1:

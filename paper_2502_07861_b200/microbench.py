@@ -29,8 +29,15 @@ def _peaks():
 
 
 def run_decode(a):
-    """Decode attention over caches loaded directly at level T (the decode-sweep shape)."""
-    B, H, g, d, Lc, T = a.batch, a.kv_heads, a.group, a.head_dim, a.cache_len, a.levels
+    print(json.dumps(decode_case(a.batch, a.kv_heads, a.group, a.head_dim, a.cache_len, a.levels, iters=a.iters,
+                                 max_layers=a.max_layers, two_instance=a.two_instance, splits=a.splits)))
+
+
+def decode_case(B, H, g, d, Lc, T, iters=50, max_layers=16, two_instance=False, splits=0):
+    """Decode attention over caches loaded directly at level T (the decode-sweep shape); returns a dict."""
+    import types
+
+    a = types.SimpleNamespace(max_layers=max_layers, two_instance=two_instance, splits=splits, iters=iters)
     esz = 2
     bytes_layer = B * H * Lc * 2 * d * esz
     # enough distinct layers that a layer is evicted from L2 (126 MB) before it is read again
@@ -65,17 +72,27 @@ def run_decode(a):
     hbm, _, src = _peaks()
     gbs = bytes_layer / (us * 1e-6) / 1e9
     st = ctx.stats()
-    print(json.dumps(dict(kernel="decode_two_instance" if a.two_instance else "decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
-                          layers_cycled=n_layers, splits=a.splits, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
-                          peak_gbs=hbm, frac=gbs / hbm, peak_source=src, device_status=st["device_status"])))
+    res = dict(kernel="decode_two_instance" if a.two_instance else "decode", batch=B, kv_heads=H, group=g, head_dim=d, cache_len=Lc, levels=T,
+               layers_cycled=n_layers, splits=a.splits, us_per_layer=us, algorithmic_bytes=bytes_layer, achieved_gbs=gbs,
+               peak_gbs=hbm, frac=gbs / hbm, peak_source=src, device_status=st["device_status"])
     ctx.close()
+    del K, V, ctx
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_compress(a):
-    """append + compress of `streams` streams (one layer), timed per kernel class."""
-    S, d, n, t, T = a.streams, a.head_dim, a.context, a.block, a.levels
+    print(json.dumps(compress_case(a.streams, a.head_dim, a.context, a.block, a.levels, iters=a.iters, gram_path=a.gram_path,
+                                   c_override=a.c_override, outliers=a.outliers, window=a.window)))
+
+
+def compress_case(S, d, n, t, T, iters=10, gram_path=0, c_override=0.0, outliers=1, window=0):
+    """append + compress of `S` streams (one layer), timed per kernel class; returns a dict."""
+    import types
+
+    a = types.SimpleNamespace(iters=iters, gram_path=gram_path, c_override=c_override, outliers=outliers)
     ctx = bk.Context(n_seqs=1, n_layers=1, n_kv_heads=S, n_q_heads=S, head_dim=d, dtype="bf16", block=t, levels=T,
-                     max_tokens=n, gram_path=a.gram_path, c_override=a.c_override)
+                     max_tokens=n, gram_path=a.gram_path, c_override=a.c_override, recent_window=window)
     K = torch.randn(1, S, n, d, device="cuda", dtype=torch.float32)
     if a.outliers:
         K[..., :4] *= 10.0
@@ -98,7 +115,7 @@ def run_compress(a):
         torch.cuda.synchronize()
         tot += e0.elapsed_time(e1)
     prof = ctx.profile_read()
-    n_calls = S * sum((n // t) >> l for l in range(T))
+    n_calls = S * sum(((n - window) // t) >> l for l in range(T))
     flop = n_calls * 2.0 * (t * (t - 1) / 2.0) * 2.0 * d
     gw_n, gw_ms = prof["gram_walk"]
     cp_n, cp_ms = prof["compact"]
@@ -107,14 +124,17 @@ def run_compress(a):
     cp_bytes = n_calls * ((t // 2) * (4 * d * 2 + 8 + 16) + t)   # rows, position, norms per survivor, sign bytes
     cp_gbs = cp_bytes * a.iters / (cp_ms * 1e-3) / 1e9 if cp_ms else 0.0
     st = ctx.stats()
-    print(json.dumps(dict(kernel="compress", streams=S, context=n, block=t, levels=T, calls=n_calls,
-                          compress_ms=tot / a.iters, gram_walk_ms=gw_ms / a.iters, gram_walk_launches=gw_n // a.iters,
-                          gram_walk_tflops=tfl, tensor_peak=tf, tensor_frac=tfl / tf,
-                          compact_ms=cp_ms / a.iters, compact_gbs=cp_gbs, hbm_peak=hbm, compact_frac=cp_gbs / hbm,
-                          radii_ms=prof["radii"][1] / a.iters, bookkeeping_ms=prof["bookkeeping"][1] / a.iters,
-                          token_heads_per_s=S * n / (tot / a.iters * 1e-3), walk_fails=st["walk_fails"],
-                          device_status=st["device_status"], peak_source=src)))
+    res = dict(kernel="compress", streams=S, context=n, block=t, levels=T, recent_window=window, calls=n_calls,
+               compress_ms=tot / a.iters, gram_walk_ms=gw_ms / a.iters, gram_walk_launches=gw_n // a.iters,
+               gram_walk_tflops=tfl, tensor_peak=tf, tensor_frac=tfl / tf,
+               compact_ms=cp_ms / a.iters, compact_gbs=cp_gbs, hbm_peak=hbm, compact_frac=cp_gbs / hbm,
+               radii_ms=prof["radii"][1] / a.iters, bookkeeping_ms=prof["bookkeeping"][1] / a.iters,
+               token_heads_per_s=S * n / (tot / a.iters * 1e-3), walk_fails=st["walk_fails"],
+               walk_kernel=st["walk_kernel"], device_status=st["device_status"], peak_source=src)
     ctx.close()
+    del K, V, ctx, flush
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_bucket(a):
@@ -194,6 +214,7 @@ def main():
     c.add_argument("--gram-path", type=int, default=0)
     c.add_argument("--c-override", type=float, default=0.0)
     c.add_argument("--outliers", type=int, default=1)
+    c.add_argument("--window", type=int, default=0, help="recent window W (tokens kept out of the calls)")
     b = sub.add_parser("bucket")
     b.add_argument("--streams", type=int, default=8)
     b.add_argument("--head-dim", type=int, default=128)
