@@ -594,17 +594,18 @@ static int run_plan(balancekv_ctx* c, Plan& P, cudaStream_t st) {
       if (c->use_tc) {
         ProfScope ps(c, 2, st);
         BKV_CUDA(launch_walk_tc(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
-                                c->dbg_p, c->d_fail, c->d_status, c->tmaps, nullptr, st));
+                                c->dbg_p, c->d_fail, c->d_status, c->tmaps, c, st));   // selection + compaction fused at the tail
       } else {
         ProfScope ps(c, 2, st);
         BKV_CUDA(launch_walk_simt(G, c->A, dc, n, l, c->d_stats, c->d_tokshift, c->d_eta, c->dbg_eta, c->dbg_S,
                                   c->dbg_p, c->d_fail, st));
       }
-      {
+      if (!c->use_tc) {
         ProfScope ps(c, 3, st);
         BKV_CUDA(launch_compact(G, c->A, dc, n, l, c->d_eta, st));
+        c->kernels_launched++;
       }
-      c->kernels_launched += 2;
+      c->kernels_launched++;
       c->calls_run += n;
     }
   }

@@ -214,12 +214,110 @@ struct Smem {
 };
 constexpr int kMaxSweeps = kTile + 2;
 
+// Output of Algorithm 2 completed to exactly t/2 tokens (the implementation note of Appendix B:
+// "strictly select n/2"), and Algorithm 3's C^{i+1} <- C^{i+1} + SoftmaxBalance(C^i): the smaller
+// sign class (ties: +1) plus the latest tokens of the other class, in stream order, copied to the
+// call's destination rows with their positions and norms.  Runs at the tail of the call's CTA, whose
+// operand slots are idle by then: `scratch` holds the kept positions.  The rows were read by this
+// CTA microseconds ago and come from L2.  All kThreads threads take part.
+__device__ inline void select_and_compact(const Geom& G, const Arena& A, const CallDesc& C, const int8_t* eta8, int* scratch) {
+  const int t = G.t, half = t / 2;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kScan = 512;                       // scanning threads (warps 0-15)
+  int* warp_sums = scratch;                        // [16] + [16]
+  int* kept_pos = scratch + 64;                    // [t/2]
+  const int ipt = (t + kScan - 1) / kScan;         // consecutive tokens per scanning thread (<= 8)
+  const int j0 = tid * ipt;
+  int plus = 0;
+  if (tid < kScan)
+    for (int i = 0; i < ipt; ++i) plus += (j0 + i < t && eta8[j0 + i] > 0) ? 1 : 0;
+  // exclusive scan of `plus` over the scanning threads
+  int inc = plus;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  if (tid < kScan && lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  int base = 0, total_plus = 0;
+#pragma unroll
+  for (int w = 0; w < kScan / 32; ++w) {
+    const int sv = warp_sums[w];
+    if (w < warp) base += sv;
+    total_plus += sv;
+  }
+  const int plus_before = base + inc - plus;
+  const int keep_sign = (total_plus <= t - total_plus) ? 1 : -1;
+  const int have = keep_sign > 0 ? total_plus : t - total_plus;
+  const int first_other_kept = (t - have) - (half - have);   // rank (in stream order) from which the other class is kept
+  int other_rank = keep_sign > 0 ? (min(j0, t) - plus_before) : plus_before;
+  int keep_cnt = 0;
+  unsigned mask = 0;
+  if (tid < kScan)
+    for (int i = 0; i < ipt; ++i) {
+      const int j = j0 + i;
+      if (j >= t) break;
+      const bool mine = (eta8[j] > 0) == (keep_sign > 0);
+      bool keep = mine;
+      if (!mine) { keep = other_rank >= first_other_kept; ++other_rank; }
+      if (keep) { mask |= 1u << i; ++keep_cnt; }
+    }
+  inc = keep_cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  if (tid < kScan && lane == 31) warp_sums[16 + warp] = inc;
+  __syncthreads();
+  int pos = inc - keep_cnt;
+#pragma unroll
+  for (int w = 0; w < kScan / 32; ++w)
+    if (w < warp) pos += warp_sums[16 + w];
+  if (tid < kScan)
+    for (int i = 0; i < ipt; ++i)
+      if (mask & (1u << i)) kept_pos[pos++] = j0 + i;
+  __syncthreads();
+  // copy: a survivor row of K and of V is 2 x 16 chunks of 16 bytes; eight loads in flight per thread.
+  // (All CTAs of a wave reach this point together, so the copy runs at the chip's memory bandwidth
+  // whichever engine moves the bytes; the bulk-copy engine was measured and is no faster.)
+  const uint4* Ks = reinterpret_cast<const uint4*>(A.K) + (size_t)C.src_row * 16;
+  const uint4* Vs = reinterpret_cast<const uint4*>(A.V) + (size_t)C.src_row * 16;
+  uint4* Kd = reinterpret_cast<uint4*>(A.K) + (size_t)C.dst_row * 16;
+  uint4* Vd = reinterpret_cast<uint4*>(A.V) + (size_t)C.dst_row * 16;
+  const int items = half * 32;
+  for (int i0 = tid; i0 < items; i0 += 8 * kThreads) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kThreads;
+      if (i < items) {
+        const int o = i >> 5, c = i & 31;
+        v[u] = (c < 16 ? Ks : Vs)[(size_t)kept_pos[o] * 16 + (c & 15)];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kThreads;
+      if (i < items) {
+        const int o = i >> 5, c = i & 31;
+        (c < 16 ? Kd : Vd)[(size_t)o * 16 + (c & 15)] = v[u];
+      }
+    }
+  }
+  for (int o = tid; o < half; o += kThreads) {
+    A.idx[C.dst_row + o] = A.idx[C.src_row + kept_pos[o]];
+    if (A.nrm) A.nrm[C.dst_row + o] = A.nrm[C.src_row + kept_pos[o]];
+  }
+}
+
 template <bool kCenter>
 __global__ void __launch_bounds__(kThreads, 1)
 walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const CallStat* __restrict__ stats,
                const float* __restrict__ tok_shift, int8_t* __restrict__ eta_out, int8_t* __restrict__ dbg_eta,
                float* __restrict__ dbg_S, float* __restrict__ dbg_p, unsigned long long* __restrict__ fail_count,
-               int* __restrict__ status, const float2* __restrict__ row_norms,
+               int* __restrict__ status, const float2* __restrict__ row_norms, const Arena A,
                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -557,13 +655,14 @@ walk_tc_kernel(Geom G, const CallDesc* __restrict__ calls, int level, const Call
       eta_out[(size_t)call * t + i] = e;
       if (C.dbg_off >= 0) dbg_eta[C.dbg_off + i] = e;
     }
+    if (A.K) select_and_compact(G, A, C, eta8, reinterpret_cast<int*>(sm));
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
-size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 9 + 2 * (kEpiGroups - 1) * kTile * 4 + 256; }
+size_t tc_smem_bytes(int t) { return 1024 + Smem::kTilesEnd + (size_t)t * 9 + 2 * (kEpiGroups - 1) * kTile * 4 + 512; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -612,17 +711,19 @@ void walk_tc_release(void* tmaps) { delete static_cast<TensorMaps*>(tmaps); }
 cudaError_t launch_walk_tc(const Geom& G, const Arena& A, const CallDesc* calls, int n_calls, int level,
                            const CallStat* stats, const float* tok_shift, int8_t* eta, int8_t* dbg_eta,
                            float* dbg_S, float* dbg_p, unsigned long long* fail_count, int* status,
-                           const void* tmaps, const void*, cudaStream_t st) {
+                           const void* tmaps, const void* fuse_compaction, cudaStream_t st) {
   if (n_calls <= 0) return cudaSuccess;
   if (!tmaps) return cudaErrorInvalidValue;
   const TensorMaps* tm = static_cast<const TensorMaps*>(tmaps);
   const size_t smem = tc_smem_bytes(G.t);
+  Arena Af = A;                       // K == nullptr: leave selection and compaction to the separate kernel
+  if (!fuse_compaction) Af.K = nullptr;
   if (G.center_keys)
     walk_tc_kernel<true><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
-                                                          fail_count, status, G.center_keys ? nullptr : A.nrm, tm->k, tm->v);
+                                                          fail_count, status, G.center_keys ? nullptr : A.nrm, Af, tm->k, tm->v);
   else
     walk_tc_kernel<false><<<n_calls, kThreads, smem, st>>>(G, calls, level, stats, tok_shift, eta, dbg_eta, dbg_S, dbg_p,
-                                                           fail_count, status, G.center_keys ? nullptr : A.nrm, tm->k, tm->v);
+                                                           fail_count, status, G.center_keys ? nullptr : A.nrm, Af, tm->k, tm->v);
   return cudaGetLastError();
 }
 
