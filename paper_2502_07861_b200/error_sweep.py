@@ -5,6 +5,7 @@ keys and values instead of the paper's prompts.
 
     python -m paper_2502_07861_b200.error_sweep --recipe clustered --n 8192 --blocks 64,256 --levels 1,2,3 --seeds 5
     python -m paper_2502_07861_b200.error_sweep --recipe clustered_norms --buckets 4 --n 16384 --blocks 64,256 --levels 1,2 --seeds 5
+    python -m paper_2502_07861_b200.error_sweep --recipe clustered_shifted --center-keys 1        (key mean shift ON; 0: OFF)
 
 Everything runs through the library: BalanceKV = append + compress + decode; uniform sampling = a
 cache loaded directly at level T with a random subset and weights 2^T; exact = a context with T = 0.
@@ -23,7 +24,7 @@ from . import binding as bk
 def make_kv(recipe, seed, H, n, d):
     """bf16 K, V [1, H, n, d] on the device."""
     g = torch.Generator(device="cuda").manual_seed(seed)
-    if recipe in ("clustered", "clustered_norms"):
+    if recipe in ("clustered", "clustered_norms", "clustered_shifted"):
         # near-duplicate keys on a few equal-norm centres, values tied to the cluster: the case in
         # which a balanced half beats a random half
         unit = lambda a: a / a.norm(dim=-1, keepdim=True)
@@ -36,6 +37,13 @@ def make_kv(recipe, seed, H, n, d):
             # value norms spread over three octaves: the case Algorithm 1's buckets are made for
             V = V * torch.exp2(-3.0 * torch.rand(H, n, 1, device="cuda", generator=g))
         Q = 0.5 * (centres[:, :4] + centres[:, 4:])                       # [H, 4, d] queries between two clusters
+        if recipe == "clustered_shifted":
+            # all keys share a large mean (as the paper observes for LLM keys, Appendix B.5): the case the
+            # mean shift before compression is made for.  The queries stay orthogonal to the mean, so exact
+            # attention is that of the unshifted keys.
+            mean = 8.0 * unit(torch.randn(H, 1, d, device="cuda", generator=g))
+            Q = Q - (Q * mean).sum(-1, keepdim=True) * mean / 64.0
+            K = K + mean
     else:
         mu = 0.5 * torch.randn(H, 1, d, device="cuda", generator=g)
         s = torch.ones(H, 1, d, device="cuda")
@@ -100,7 +108,7 @@ def run_point(recipe, seed, H, n, d, t, T, c_small, center, buckets=0):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--recipe", default="clustered", choices=("clustered", "clustered_norms", "llama"))
+    ap.add_argument("--recipe", default="clustered", choices=("clustered", "clustered_norms", "clustered_shifted", "llama"))
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--heads", type=int, default=4)
     ap.add_argument("--head-dim", type=int, default=128)
