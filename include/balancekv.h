@@ -277,6 +277,24 @@ int balancekv_stream_append_layer_bucketed(balancekv_ctx* ctx, int layer0, int n
                                            const void* V, int n_tokens, float erase_ratio, int8_t* token_slot,
                                            int32_t* counts_host, void* stream);
 
+/* The augmented BalanceKV of Section 4.3: tokens whose keys are strongly anti-correlated with the
+ * rest are preserved exactly, the standard procedure runs on the others.  The paper gives neither
+ * the measure nor a threshold; here token j of the appended block is preserved when the cosine
+ * between its key and the block's mean key (per stream) is at most tau,
+ *   <k_j, kbar> <= tau ||k_j|| ||kbar||,   -1 <= tau <= 1 (tau = -1 preserves nothing but exact
+ * opposites; a zero key or mean counts as cosine 0),
+ * compared in fp32.  The caller dedicates two consecutive layer slots to one model layer: slot
+ * layer0 receives the preserved rows and is never compressed (use balancekv_compress_layer on slot
+ * layer0 + 1 only), slot layer0 + 1 receives the rest in stream order and is an ordinary BalanceKV
+ * stream.  balancekv_decode_attn_merged over both slots on both sides is the estimator of
+ * Theorem 3.3 over the union: preserved tokens weigh 1, so the weights still sum to the tokens seen.
+ * K, V: [n_seqs, n_kv_heads, n_tokens, head_dim] device; token_slot (device, may be NULL): int8 per
+ * row, 0 = preserved, 1 = the rest; counts_host (host, may be NULL): per stream {preserved, rest,
+ * dropped = 0}.  The stored original position of a row is its position in its slot's own stream.
+ * Synchronises `stream` once, like the bucketed append.  Errors as for the bucketed append. */
+int balancekv_stream_append_layer_preserving(balancekv_ctx* ctx, int layer0, const void* K, const void* V, int n_tokens,
+                                             float tau, int8_t* token_slot, int32_t* counts_host, void* stream);
+
 /* Kernel timing for roofline reports.  While enabled, every launch of the kernel classes
  * below is bracketed by CUDA events on its launch stream (at most 8192 launches between two
  * reads; later ones are not recorded).  balancekv_profile_read synchronises the device and

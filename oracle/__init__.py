@@ -19,3 +19,4 @@ from .binding import (  # noqa: F401
     weighted_sums,
 )
 from .bucketing import NO_BUCKET, BucketedOracle, value_bucket  # noqa: F401,E402
+from .preserving import PreservingOracle, anticorrelated  # noqa: F401,E402

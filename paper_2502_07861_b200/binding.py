@@ -24,7 +24,7 @@ EXPORTS = [
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
     "balancekv_decode_attn_two", "balancekv_decode_attn_merged", "balancekv_stream_append_bucketed",
-    "balancekv_stream_append_layer_bucketed", "balancekv_debug_set_status", "balancekv_decode_attn_static_status",
+    "balancekv_stream_append_layer_bucketed", "balancekv_stream_append_layer_preserving", "balancekv_debug_set_status", "balancekv_decode_attn_static_status",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -95,6 +95,7 @@ def load():
     lib.balancekv_profile_read.argtypes = [vp, vp]
     lib.balancekv_stream_append_bucketed.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
     lib.balancekv_stream_append_layer_bucketed.argtypes = [vp, ci, ci, ci, vp, vp, ci, C.c_float, vp, vp, vp]
+    lib.balancekv_stream_append_layer_preserving.argtypes = [vp, ci, vp, vp, ci, C.c_float, vp, vp, vp]
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     lib.balancekv_decode_attn_static_status.argtypes = [vp, vp]
     lib.balancekv_debug_set_status.argtypes = [vp, ci]
@@ -243,6 +244,22 @@ class Context:
             self._h, layer0, n_buckets, i_top, self._dev(K, "K"), self._dev(V, "V"), K.shape[2], float(erase_ratio),
             slots.data_ptr() if want_slots else None, counts.ctypes.data, _stream_ptr(stream)),
             "balancekv_stream_append_layer_bucketed")
+        return (counts, slots) if want_slots else counts
+
+    def stream_append_layer_preserving(self, layer0, K, V, tau, want_slots=False, stream=None):
+        """Section 4.3's augmented variant: rows whose key has cosine <= tau with the block's mean key go to slot
+        layer0 (kept exactly), the rest to slot layer0 + 1.  Returns counts [B*H, 3] (preserved, rest, dropped)
+        and, if asked, the int8 slot of every row [B, H, n]."""
+        import numpy as np
+        import torch
+
+        assert K.shape == V.shape and K.dim() == 4
+        counts = np.zeros((K.shape[0] * K.shape[1], 3), np.int32)
+        slots = torch.empty(K.shape[:3], dtype=torch.int8, device=K.device) if want_slots else None
+        _check(self.lib.balancekv_stream_append_layer_preserving(
+            self._h, layer0, self._dev(K, "K"), self._dev(V, "V"), K.shape[2], float(tau),
+            slots.data_ptr() if want_slots else None, counts.ctypes.data, _stream_ptr(stream)),
+            "balancekv_stream_append_layer_preserving")
         return (counts, slots) if want_slots else counts
 
     def stream_append_bucketed(self, seq, layer0, n_buckets, i_top, kv_head, K, V, erase_ratio=0.0, want_slots=False,

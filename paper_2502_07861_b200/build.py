@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbalancekv.so")
 SOURCES = ["api.cu", "kernels_misc.cu", "kernels_walk_simt.cu", "kernels_walk_tc.cu", "kernels_compact.cu",
-           "kernels_decode.cu", "kernels_decode_mma.cu", "decode_static.cu", "kernels_bucket.cu"]
+           "kernels_decode.cu", "kernels_decode_mma.cu", "decode_static.cu", "kernels_bucket.cu", "kernels_anticorr.cu"]
 HEADERS = ["common.cuh", "sched.h", os.path.join("..", "..", "include", "balancekv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]

@@ -145,6 +145,10 @@ struct balancekv_ctx {
   BucketOut* bkt_out_host = nullptr;    // pinned
   size_t bkt_rows = 0, bkt_streams = 0;
   int64_t bucket_dropped = 0;
+  // preservation of anti-correlated keys: column sums / mean scratch and the class of every row
+  float* acr_scratch = nullptr;
+  int8_t* acr_cls = nullptr;
+  size_t acr_floats = 0, acr_rows = 0;
 
   // optional per-class kernel timing
   unsigned profiling = 0;                   // bit per kernel class
@@ -388,7 +392,7 @@ int balancekv_destroy(balancekv_ctx* c) {
                   c->view_idx, c->bounce_K, c->bounce_V, c->bounce_q, c->bounce_out, c->step_dev_in, c->step_dev_out, c->two_acc, c->two_ml, c->two_scratch, c->unit_V};
   for (void* p : ptrs)
     if (p) cudaFree(p);
-  void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out, c->bkt_chunk_cnt};
+  void* bkt[] = {c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_vmax_bits, c->bkt_out, c->bkt_chunk_cnt, c->acr_scratch, c->acr_cls};
   for (void* p : bkt)
     if (p) cudaFree(p);
   if (c->bkt_out_host) cudaFreeHost(c->bkt_out_host);
@@ -1034,7 +1038,8 @@ int balancekv_debug_call(balancekv_ctx* c, int seq, int layer, int kv_head, int 
 // consecutively in K, V.  Slot layer0 + b is the instance of bucket index i_top - b.
 static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<int, int>>& heads, int layer0,
                                 int n_buckets, int i_top, const void* K, const void* V, int n, float rho,
-                                int8_t* token_slot, int32_t* counts_host, cudaStream_t st) {
+                                int8_t* token_slot, int32_t* counts_host, cudaStream_t st, bool preserve = false,
+                                float tau = 0.f) {
   const balancekv_config& f = c->cfg;
   const Layout& Lo = c->Lo;
   if (!K || !V || n < 1 || n > (1 << 22) || !aligned16(K) || !aligned16(V)) return BALANCEKV_E_INVAL;
@@ -1077,10 +1082,29 @@ static int append_bucketed_impl(balancekv_ctx* c, const std::vector<std::pair<in
   void* d_in = nullptr;
   int rc = ring_push(c, in.data(), in.size() * sizeof(BucketIn), st, &d_in);
   if (rc) return rc;
+  const int8_t* forced = nullptr;
+  if (preserve) {
+    // slot of every row from its key's cosine with the block's mean key instead of from its value norm
+    const size_t need_f = anticorr_scratch_floats(n_sl, n, f.head_dim), need_c = (size_t)n_sl * n;
+    if (need_f > c->acr_floats || need_c > c->acr_rows) {
+      BKV_CUDA(cudaStreamSynchronize(st));
+      if (c->acr_scratch) cudaFree(c->acr_scratch);
+      if (c->acr_cls) cudaFree(c->acr_cls);
+      c->acr_scratch = nullptr; c->acr_cls = nullptr;
+      c->acr_floats = std::max(c->acr_floats, need_f);
+      c->acr_rows = std::max(c->acr_rows, need_c);
+      BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->acr_scratch), sizeof(float) * c->acr_floats));
+      BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->acr_cls), c->acr_rows));
+    }
+    ProfScope ps(c, 0, st);
+    BKV_CUDA(launch_anticorr_classes(c->G, K, n_sl, n, tau, c->acr_scratch, c->acr_cls, st));
+    c->kernels_launched += 3;
+    forced = c->acr_cls;
+  }
   {
     ProfScope ps(c, 0, st);
     BKV_CUDA(launch_bucket_route(c->G, V, n_sl, n, n_buckets, i_top, rho * rho, static_cast<const BucketIn*>(d_in),
-                                 c->bkt_vmax_bits, c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_chunk_cnt, c->bkt_out, st));
+                                 c->bkt_vmax_bits, c->bkt_ns, c->bkt_slot, c->bkt_rank, c->bkt_chunk_cnt, c->bkt_out, forced, st));
   }
   c->kernels_launched += 3;
   BKV_CUDA(cudaMemcpyAsync(c->bkt_out_host, c->bkt_out, sizeof(BucketOut) * n_sl, cudaMemcpyDeviceToHost, st));
@@ -1165,6 +1189,16 @@ int balancekv_stream_append_layer_bucketed(balancekv_ctx* c, int layer0, int n_b
     for (int h = 0; h < c->cfg.n_kv_heads; ++h) heads.push_back({s, h});
   return append_bucketed_impl(c, heads, layer0, n_buckets, i_top, K, V, n_tokens, erase_ratio, token_slot, counts_host,
                               static_cast<cudaStream_t>(stream));
+}
+
+int balancekv_stream_append_layer_preserving(balancekv_ctx* c, int layer0, const void* K, const void* V, int n_tokens,
+                                             float tau, int8_t* token_slot, int32_t* counts_host, void* stream) {
+  if (!c || !(tau >= -1.f) || tau > 1.f) return BALANCEKV_E_INVAL;
+  std::vector<std::pair<int, int>> heads;
+  for (int s = 0; s < c->cfg.n_seqs; ++s)
+    for (int h = 0; h < c->cfg.n_kv_heads; ++h) heads.push_back({s, h});
+  return append_bucketed_impl(c, heads, layer0, 2, 0, K, V, n_tokens, 0.f, token_slot, counts_host,
+                              static_cast<cudaStream_t>(stream), true, tau);
 }
 
 int balancekv_reset(balancekv_ctx* c, void* stream) {

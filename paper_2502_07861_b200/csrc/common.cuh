@@ -187,7 +187,10 @@ int bucket_scan_chunks(int n);
 size_t bucket_chunk_count_ints(int n_sl, int n);   // ints of the per-chunk count table of the routing pass
 cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, int n_buckets, int i_top, float rho2,
                                 const BucketIn* in, unsigned* vmax2_bits, float* ns, int8_t* slot, int32_t* rank,
-                                int32_t* chunk_cnt, BucketOut* out, cudaStream_t st);
+                                int32_t* chunk_cnt, BucketOut* out, const int8_t* forced_slot, cudaStream_t st);
+size_t anticorr_scratch_floats(int n_sl, int n, int d);
+cudaError_t launch_anticorr_classes(const Geom& G, const void* K, int n_sl, int n, float tau, float* scratch, int8_t* cls,
+                                    cudaStream_t st);
 cudaError_t launch_bucket_scatter(const Geom& G, const Arena& A, const void* K, const void* V, int n_sl, int n,
                                   int n_buckets, const int8_t* slot, const int32_t* rank, const int32_t* chunk_base,
                                   const float* ns, const BucketDst* dst, cudaStream_t st);

@@ -111,7 +111,7 @@ __device__ inline int erase_index(float rho2, const BucketIn& in, unsigned vmax2
 __global__ void __launch_bounds__(kScanThreads)
 bucket_scan_kernel(const float* __restrict__ ns, int n, int n_chunks, int n_buckets, int i_top, float rho2,
                    const BucketIn* __restrict__ in, const unsigned* __restrict__ vmax2_bits, int8_t* __restrict__ slot,
-                   int32_t* __restrict__ rank, int32_t* __restrict__ chunk_cnt) {
+                   int32_t* __restrict__ rank, int32_t* __restrict__ chunk_cnt, const int8_t* __restrict__ forced) {
   constexpr int kWarps = kScanThreads / 32, kRounds = kScanChunk / kScanThreads;
   __shared__ int warp_tot[kCountCols][kWarps];
   const int sl = blockIdx.y, chunk = blockIdx.x;
@@ -133,7 +133,9 @@ bucket_scan_kernel(const float* __restrict__ ns, int n, int n_chunks, int n_buck
 #pragma unroll
   for (int u = 0; u < kRounds; ++u) {
     int b = -3;                                          // past the end of the block
-    if (x[u] >= 0.f) {
+    if (x[u] >= 0.f && forced) {
+      b = forced[base + j0 + u * 32 + lane];             // the slot was decided elsewhere (not by the value norm)
+    } else if (x[u] >= 0.f) {
       b = kMaxBuckets;                                   // dropped
       if (x[u] > 0.f) {
         const int i = bucket_of(x[u]);
@@ -255,7 +257,7 @@ size_t bucket_chunk_count_ints(int n_sl, int n) { return (size_t)n_sl * bucket_s
 
 cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, int n_buckets, int i_top, float rho2,
                                 const BucketIn* in, unsigned* vmax2_bits, float* ns, int8_t* slot, int32_t* rank,
-                                int32_t* chunk_cnt, BucketOut* out, cudaStream_t st) {
+                                int32_t* chunk_cnt, BucketOut* out, const int8_t* forced_slot, cudaStream_t st) {
   const int chunks = G.d * (G.is_bf16 ? 2 : 4) / 16;
   cudaError_t e = cudaMemsetAsync(vmax2_bits, 0, sizeof(unsigned) * n_sl, st);
   if (e != cudaSuccess) return e;
@@ -264,7 +266,7 @@ cudaError_t launch_bucket_route(const Geom& G, const void* V, int n_sl, int n, i
   else bucket_norms_kernel<false><<<grid, 256, 0, st>>>(V, n, chunks, ns, vmax2_bits);
   const int n_chunks = bucket_scan_chunks(n);
   bucket_scan_kernel<<<dim3(n_chunks, n_sl), kScanThreads, 0, st>>>(ns, n, n_chunks, n_buckets, i_top, rho2, in, vmax2_bits,
-                                                                   slot, rank, chunk_cnt);
+                                                                   slot, rank, chunk_cnt, forced_slot);
   bucket_prefix_kernel<<<n_sl, kCountCols * 32, 0, st>>>(n_chunks, rho2, in, vmax2_bits, chunk_cnt, out);
   return cudaGetLastError();
 }
