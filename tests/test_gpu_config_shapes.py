@@ -115,12 +115,28 @@ def test_14b_shape_three_levels_window_student_t(cuda_lib):
     for c0 in range(0, n, chunk):
         K, V = _gen(4000 + c0 // chunk, B, H, chunk, d, "student_t")
         if c0 == 0:
-            first = (_f64(K[5, 2, :t]), _f64(V[5, 2, :t]))
+            first = (_f64(K[5, 2, :4 * t]), _f64(V[5, 2, :4 * t]))        # the first four blocks of one stream
         ctx.stream_append_layer(0, K, V)
         ctx.compress()
     st = ctx.stats()
     assert st["device_status"] == 0 and st["calls_run"] == B * H * (63 + 31 + 15)
-    _check_call(ctx, OracleParams(d=d, t=t, T=T, W=W, layer=0, head=2, max_tokens=n, seed=1 + 5), *first, 5, 0, 2, 0, 0)
+    # one teacher-forced chain through every level: level-0 calls 0..3 of a stream, the level-1 calls 0 and 1 on
+    # their survivors, the level-2 call 0 on theirs; its survivors are the first rows of C^3
+    P = OracleParams(d=d, t=t, T=T, W=W, layer=0, head=2, max_tokens=n, seed=1 + 5)
+    Kl, Vl, pos = [first[0][i * t:(i + 1) * t] for i in range(4)], [first[1][i * t:(i + 1) * t] for i in range(4)], \
+        [np.arange(i * t, (i + 1) * t) for i in range(4)]
+    for level in range(T):
+        Kn, Vn, pn = [], [], []
+        for o in range(len(Kl)):
+            r = _check_call(ctx, P, Kl[o], Vl[o], 5, 0, 2, level, o)
+            assert len(r["kept"]) == t // 2
+            Kn.append(Kl[o][r["kept"]]); Vn.append(Vl[o][r["kept"]]); pn.append(pos[o][r["kept"]])
+        Kl = [np.concatenate(Kn[i:i + 2]) for i in range(0, len(Kn), 2)]
+        Vl = [np.concatenate(Vn[i:i + 2]) for i in range(0, len(Vn), 2)]
+        pos = [np.concatenate(pn[i:i + 2]) for i in range(0, len(pn), 2)]
+    Kc, Vc, w, idx = ctx.cache_view(5, 0, 2)
+    assert np.array_equal(idx[:t // 2].cpu().numpy(), pos[0]) and torch.all(w[:t // 2] == 8.0)
+    assert np.array_equal(_f64(Kc[:t // 2]), Kl[0]) and np.array_equal(_f64(Vc[:t // 2]), Vl[0])
     # stored per stream: 15*512 rows at weight 8, 512 at 4, 512 at 2, 896 + the window of 128 at 1
     for b in (0, 7):
         for h in (0, 4):
