@@ -30,10 +30,10 @@ def _peaks():
 
 def run_decode(a):
     print(json.dumps(decode_case(a.batch, a.kv_heads, a.group, a.head_dim, a.cache_len, a.levels, iters=a.iters,
-                                 max_layers=a.max_layers, two_instance=a.two_instance, splits=a.splits)))
+                                 max_layers=a.max_layers, two_instance=a.two_instance, splits=a.splits, gram_path=a.gram_path)))
 
 
-def decode_case(B, H, g, d, Lc, T, iters=50, max_layers=16, two_instance=False, splits=0):
+def decode_case(B, H, g, d, Lc, T, iters=50, max_layers=16, two_instance=False, splits=0, gram_path=0):
     """Decode attention over caches loaded directly at level T (the decode-sweep shape); returns a dict."""
     import types
 
@@ -46,7 +46,7 @@ def decode_case(B, H, g, d, Lc, T, iters=50, max_layers=16, two_instance=False, 
         n_layers += n_layers % 2
         bytes_layer = bytes_layer * 3 // 2      # K and V of the numerator slot, K of the denominator slot
     ctx = bk.Context(n_seqs=B, n_layers=n_layers, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64,
-                     levels=T, max_tokens=Lc << T, decode_splits=a.splits)
+                     levels=T, max_tokens=Lc << T, decode_splits=a.splits, gram_path=gram_path)
     K = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     V = torch.randn(B, H, Lc, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     for l in range(n_layers):
@@ -204,6 +204,7 @@ def main():
     d.add_argument("--max-layers", type=int, default=16)
     d.add_argument("--two-instance", action="store_true")
     d.add_argument("--splits", type=int, default=0, help="split-K factor (0 = automatic)")
+    d.add_argument("--gram-path", type=int, default=0, help="1: the CUDA-core decode kernel")
     c = sub.add_parser("compress")
     c.add_argument("--streams", type=int, default=8)
     c.add_argument("--head-dim", type=int, default=128)
