@@ -271,6 +271,7 @@ def main():
     ap.add_argument("--gram-path", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="skip the slices of the other configurations")
+    ap.add_argument("--decode-splits", type=int, default=0, help="split-K factor of decode attention (0 = automatic)")
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling a small case)")
     ap.add_argument("--decode-steps", type=int, default=None)
     args = ap.parse_args()
@@ -315,7 +316,8 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     ctx = bk.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, head_dim=d, dtype="bf16", block=t, levels=T,
-                     max_tokens=n_ctx + n_dec, seed=shard.walk_seed(w["walk_seed"], rank * B), gram_path=args.gram_path)
+                     max_tokens=n_ctx + n_dec, seed=shard.walk_seed(w["walk_seed"], rank * B), gram_path=args.gram_path,
+                     decode_splits=args.decode_splits)
 
     raw_stream = int(torch.cuda.current_stream().cuda_stream)
     q_list, K_list, V_list = list(q_d.unbind(0)), list(K_dec.unbind(0)), list(V_dec.unbind(0))

@@ -450,7 +450,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   // With a single split the CTA's partial is the stream's result: it stays in shared memory (behind
   // the merge buffers) and the ticket, the fences and the staging copy are skipped.
   constexpr uint32_t kMrg2Off = kWarps * kMaxGroup * PS * 4;        // behind mrg: [ways][g][PS] first-level merges
-  constexpr uint32_t kSingleOff = kMrg2Off + kWarps * PS * 4 + 512;
+  constexpr uint32_t kSingleOff = 4352 + kWarps * kMaxGroup * 32 * 16 + 4096;   // behind the merge buffers and the combine's tables
   const bool single = splits == 1;
   // Partial results: per (stream, split, head) a row of kD column sums, and behind all rows the
   // (max, sum) pairs.  Rows of 512 bytes keep the staging copy 128-byte aligned.
@@ -542,8 +542,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
   float* cL = cM + kMaxGroup;                             // [g] overall sum
   float* cN = cL + kMaxGroup;                             // [g] factor of the appended token
-  float4* red = reinterpret_cast<float4*>(tiles + 4352);  // [ways - 1][g][32] partial column sums (<= 7680 bytes)
-  constexpr uint32_t kStageOff = 16384;                    // behind cm, cl, cM, cL, cN, red
+  constexpr uint32_t kStageOff = 4352 + kWarps * kMaxGroup * 32 * 16;   // behind cm, cl, cM, cL, cN and the column-sum parts
   const uint32_t part_bytes = (uint32_t)splits * g * kD * sizeof(float);
   const bool staged = single || part_bytes <= kStages * kStageBytes - kStageOff;
   const float* sp_s = reinterpret_cast<const float*>(tiles + (single ? kSingleOff : kStageOff));
@@ -651,90 +650,82 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     if (lane == 0) { cM[h] = M; cL[h] = L; cN[h] = fN; }
   }
   __syncthreads();
-  // Column sums over the splits: item (mh, mw) takes the splits mw, mw + ways, ... of its head, lane =
-  // 4 consecutive columns; the ways meet in shared memory.
-  float4 accs[kHeadsPer];
+  // Column sums over the splits: warp w takes the splits w, w + kWarps, ... for every head (lane = 4
+  // consecutive columns, one accumulator per head: the chain per thread is splits / kWarps long and the
+  // heads' loads are independent); the warps' parts meet in shared memory, where warp h sums head h.
+  float4 acc[kMaxGroup];
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
   bool landed = true;
   if (staged && !single) {
     if (lane == 0) landed = mbar_wait(cbar, 0u);
     landed = __shfl_sync(0xffffffffu, landed, 0);
     __syncwarp();
   }
-#pragma unroll
-  for (int k = 0; k < kHeadsPer; ++k) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int r = warp + k * kWarps;
-    if (r < n_r) {
-      int ih = mh, iw = mw;
-      if (k > 0) { ih = r; iw = 0; }            // more heads than warps: ways = 1
-      const size_t row_stride = (size_t)g * kD, step = (size_t)ways * row_stride;
-      const float* fac = cm + ih + iw * g;
-      const int fstep = ways * g;
-      int n = iw < splits ? (splits - iw + ways - 1) / ways : 0;     // splits of this way
+  {
+    const size_t row_stride = (size_t)g * kD;
+    for (int sp_i = warp; sp_i < splits; sp_i += kWarps) {
+      const float* fac = cm + (size_t)sp_i * g;
       if (staged) {
-        const float* p = sp_s + (size_t)iw * row_stride + (size_t)ih * kD + 4 * lane;
-        for (; n >= 4; n -= 4, p += 4 * step, fac += 4 * fstep) {
-          const float4 v0 = *reinterpret_cast<const float4*>(p), v1 = *reinterpret_cast<const float4*>(p + step);
-          const float4 v2 = *reinterpret_cast<const float4*>(p + 2 * step), v3 = *reinterpret_cast<const float4*>(p + 3 * step);
-          const float f0 = fac[0], f1 = fac[fstep], f2 = fac[2 * fstep], f3 = fac[3 * fstep];
-          acc.x = fmaf(v0.x, f0, acc.x); acc.y = fmaf(v0.y, f0, acc.y); acc.z = fmaf(v0.z, f0, acc.z); acc.w = fmaf(v0.w, f0, acc.w);
-          acc.x = fmaf(v1.x, f1, acc.x); acc.y = fmaf(v1.y, f1, acc.y); acc.z = fmaf(v1.z, f1, acc.z); acc.w = fmaf(v1.w, f1, acc.w);
-          acc.x = fmaf(v2.x, f2, acc.x); acc.y = fmaf(v2.y, f2, acc.y); acc.z = fmaf(v2.z, f2, acc.z); acc.w = fmaf(v2.w, f2, acc.w);
-          acc.x = fmaf(v3.x, f3, acc.x); acc.y = fmaf(v3.y, f3, acc.y); acc.z = fmaf(v3.z, f3, acc.z); acc.w = fmaf(v3.w, f3, acc.w);
-        }
-        for (; n > 0; --n, p += step, fac += fstep) {
-          const float4 v0 = *reinterpret_cast<const float4*>(p);
-          const float f0 = fac[0];
-          acc.x = fmaf(v0.x, f0, acc.x); acc.y = fmaf(v0.y, f0, acc.y); acc.z = fmaf(v0.z, f0, acc.z); acc.w = fmaf(v0.w, f0, acc.w);
+        const float* p = sp_s + (size_t)sp_i * row_stride + 4 * lane;
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h) {
+          if (h < g) {
+            const float4 v = *reinterpret_cast<const float4*>(p + (size_t)h * kD);
+            const float f = fac[h];
+            acc[h].x = fmaf(v.x, f, acc[h].x); acc[h].y = fmaf(v.y, f, acc[h].y);
+            acc[h].z = fmaf(v.z, f, acc[h].z); acc[h].w = fmaf(v.w, f, acc[h].w);
+          }
         }
       } else {
-        const float* p = sp + (size_t)iw * row_stride + (size_t)ih * kD + 4 * lane;
-        for (; n > 0; n -= 8) {
-          float4 v[8];
+        const float* p = sp + (size_t)sp_i * row_stride + 4 * lane;
+        float4 v[kMaxGroup];
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
-            v[u] = u < n ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)u * step)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int h = 0; h < kMaxGroup; ++h)
+          v[h] = h < g ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)h * kD)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const float f = u < n ? fac[u * fstep] : 0.f;
-            acc.x = fmaf(v[u].x, f, acc.x); acc.y = fmaf(v[u].y, f, acc.y);
-            acc.z = fmaf(v[u].z, f, acc.z); acc.w = fmaf(v[u].w, f, acc.w);
+        for (int h = 0; h < kMaxGroup; ++h) {
+          if (h < g) {
+            const float f = fac[h];
+            acc[h].x = fmaf(v[h].x, f, acc[h].x); acc[h].y = fmaf(v[h].y, f, acc[h].y);
+            acc[h].z = fmaf(v[h].z, f, acc[h].z); acc[h].w = fmaf(v[h].w, f, acc[h].w);
           }
-          p += 8 * step;
-          fac += 8 * fstep;
         }
       }
-      if (iw > 0) red[((size_t)(iw - 1) * g + ih) * 32 + lane] = acc;
     }
-    accs[k] = acc;
   }
   if (!landed && lane == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
-  if (ways > 1) __syncthreads();
+  float4* red = reinterpret_cast<float4*>(tiles + 4352);  // [kWarps][g][32] partial column sums (<= 16 KB; the staged rows lie behind)
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h)
+    if (h < g) red[((size_t)warp * g + h) * 32 + lane] = acc[h];
+  __syncthreads();
 #pragma unroll
   for (int k = 0; k < kHeadsPer; ++k) {
     const int h = warp + k * kWarps;
     if (h >= g) break;
-    float4 acc = accs[k];
-    for (int w = 1; w < ways; ++w) {
-      const float4 r = red[((size_t)(w - 1) * g + h) * 32 + lane];
-      acc.x += r.x; acc.y += r.y; acc.z += r.z; acc.w += r.w;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float4 r = red[((size_t)w * g + h) * 32 + lane];
+      a.x += r.x; a.y += r.y; a.z += r.z; a.w += r.w;
     }
     const int c = 4 * lane;
     if (ap.k_new) {
       const float fN = cN[h];
       const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.y);
-      acc.x = fmaf(__bfloat162float(v01.x), fN, acc.x); acc.y = fmaf(__bfloat162float(v01.y), fN, acc.y);
-      acc.z = fmaf(__bfloat162float(v23.x), fN, acc.z); acc.w = fmaf(__bfloat162float(v23.y), fN, acc.w);
+      a.x = fmaf(__bfloat162float(v01.x), fN, a.x); a.y = fmaf(__bfloat162float(v01.y), fN, a.y);
+      a.z = fmaf(__bfloat162float(v23.x), fN, a.z); a.w = fmaf(__bfloat162float(v23.y), fN, a.w);
     }
     const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
     if (raw_acc) {
-      *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = acc;
+      *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = a;
       if (c == 0) { raw_ml[2 * qh] = cM[h]; raw_ml[2 * qh + 1] = cL[h]; }
     } else {
       const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
       __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + qh * kD + c);
-      o2[0] = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-      o2[1] = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+      o2[0] = __floats2bfloat162_rn(a.x * inv, a.y * inv);
+      o2[1] = __floats2bfloat162_rn(a.z * inv, a.w * inv);
     }
   }
   if (tid == 0 && !single) tickets[sl] = 0;   // ready for the next launch
