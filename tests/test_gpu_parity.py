@@ -289,3 +289,28 @@ def test_a_timed_out_wait_surfaces_as_an_error_code_and_reset_clears_it(cuda_lib
     ctx.decode_attn(0, q)
     assert ctx.stats()["device_status"] == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("g", [1, 2, 3, 5, 6, 7, 8])
+@pytest.mark.parametrize("splits", [1, 5, 24, 64])
+def test_decode_kernel_every_group_size_and_split_factor(cuda_lib, g, splits):
+    """The tensor-core decode kernel against the oracle's weighted attention for every group size and for split
+    factors that take each of its combine paths: a single split (no ticket), partial rows staged in shared memory,
+    and more partial rows than fit there (read from global memory: g = 8 with 24 or 64 splits).  Two levels with
+    ragged lengths, one of them shorter than a tile."""
+    B, H, d, T, n_heavy, n_tail = 1, 2, 128, 2, 2500, 37
+    ctx = cuda_lib.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64, levels=T,
+                           max_tokens=(n_heavy << T) + 64, decode_splits=splits)
+    K, V = synth.layer_kv("llama", 31, 0, B, H, n_heavy + n_tail, d, "bf16")
+    ctx.cache_load_level(0, T, to_device(K[:, :, :n_heavy], "bf16"), to_device(V[:, :, :n_heavy], "bf16"))
+    ctx.stream_append_layer(0, to_device(K[:, :, n_heavy:], "bf16"), to_device(V[:, :, n_heavy:], "bf16"))
+    w = np.concatenate([np.full(n_heavy, 4.0), np.ones(n_tail)])
+    for step in range(2):                                   # twice: the tickets and the scratch are reused
+        q = synth.queries(31, 0, step, B, H * g, d, "bf16")
+        out = ctx.decode_attn(0, to_device(q, "bf16")).float().cpu().numpy()
+        for h in range(H):
+            ref = oracle.weighted_attention(K[0, h], V[0, h], w, q[0, h * g:(h + 1) * g])
+            assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3, (g, splits, h)
+    st = ctx.stats()
+    assert st["device_status"] == 0 and st["decode_kernel"] == 2
+    ctx.close()
