@@ -135,8 +135,11 @@ int balancekv_stream_step(balancekv_ctx* ctx, int layer, const void* q, const vo
                           void* out, void* stream);
 /* Same with HOST buffers for q, k_new, v_new and out.  The inputs are read by the CPU during
  * the call (packed into a pinned staging slot of the context and sent as one transfer on a copy
- * stream of the context, which the step's kernel on `stream` waits for: the transfer of a step
- * overlaps the previous step's kernel), so the caller may reuse them as soon as the call returns; out_host is written in stream order
+ * stream of the context, so that the transfer of a step overlaps the previous step's kernel), and the
+ * caller may reuse them as soon as the call returns.  The fused step kernel is not tied to that
+ * transfer by an event: an arrival word is written behind the operands on the copy stream and the
+ * kernel waits for it (bounded like every device-side wait); where the step takes more than one
+ * launch the launches wait for the transfer through an event.  out_host is written in stream order
  * (synchronise the stream before reading it): a pinned out_host is written by the kernel itself,
  * pageable memory through a device buffer and a copy.  The first call allocates the staging buffers. */
 int balancekv_stream_step_host(balancekv_ctx* ctx, int layer, const void* q_host, const void* k_host,

@@ -10,6 +10,8 @@
 #include <utility>
 #include <vector>
 
+#include <cuda.h>
+
 #include "../../include/balancekv.h"
 #include "common.cuh"
 #include "sched.h"
@@ -35,7 +37,8 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
                                 void* out, int n_heads, int d, cudaStream_t st);
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, const int* in_flag,
+                                   int in_expect, cudaStream_t st);
 }  // namespace bkv
 
 #define BKV_CUDA(expr)                                                                    \
@@ -113,6 +116,10 @@ struct balancekv_ctx {
   size_t step_slot_bytes = 0;
   cudaEvent_t step_ev[kStepSlots] = {};
   unsigned long long step_count = 0;
+  const int* step_flag = nullptr;       // set by stream_step_host for the launch that follows: arrival flag of its operands
+  int step_expect = 0;
+  void* write_value_fn = nullptr;       // cuStreamWriteValue32, if the driver offers it
+  cudaEvent_t step_group_ev[4] = {};    // kernels of 16 consecutive host steps have finished (their slots may be reused)
   // two-instance estimator: un-normalised parts of the numerator and denominator instances, unit values
   float* two_acc = nullptr;             // [BALANCEKV_MAX_MERGE][B, Hq, d] value sums per merged slot
   float* two_ml = nullptr;              // [BALANCEKV_MAX_MERGE][B, Hq, 2] (max, sum) per merged slot
@@ -401,6 +408,8 @@ int balancekv_destroy(balancekv_ctx* c) {
   if (c->step_host) cudaFreeHost(c->step_host);
   if (c->step_copy_stream) cudaStreamDestroy(c->step_copy_stream);
   for (cudaEvent_t e : c->step_used_ev)
+    if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->step_group_ev)
     if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->step_ev)
     if (e) cudaEventDestroy(e);
@@ -731,7 +740,7 @@ int balancekv_decode_attn(balancekv_ctx* c, int layer, const void* q, void* out,
       cudaStream_t st = static_cast<cudaStream_t>(stream);
       const int early = alike && c->decode_chain && c->chain_stream == st;
       BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                      nullptr, nullptr, 0, 0, 0, alike ? hint : nullptr, early, st));
+                                      nullptr, nullptr, 0, 0, 0, alike ? hint : nullptr, early, nullptr, 0, st));
       c->decode_chain = true;
       c->chain_stream = st;
     } else
@@ -847,6 +856,22 @@ int balancekv_decode_attn_two(balancekv_ctx* c, int layer_num, int layer_den, co
   return balancekv_decode_attn_merged(c, &n, 1, &dn, 1, q, out, stream);
 }
 
+// True if balancekv_stream_step will serve this layer's step with the one fused launch.
+static bool step_can_fuse(balancekv_ctx* c, int layer) {
+  if (!c->decode_maps) return false;
+  const balancekv_config& f = c->cfg;
+  const Layout& Lo = c->Lo;
+  const std::vector<int>& streams = layer_streams(c, layer);
+  const int max_pending = Lo.T == 0 ? f.max_tokens : (f.max_pending > 0 ? std::min(f.max_pending, f.max_tokens) : f.max_tokens);
+  const StreamState& S0 = c->st[streams[0]];
+  for (int s : streams) {
+    const StreamState& S = c->st[s];
+    if (S.start0 != S0.start0 || S.len0 != S0.len0 || S.appended != S0.appended) return false;
+    if (S.appended + 1 > f.max_tokens || S.pending + 1 > max_pending || (int64_t)S.start0 + S.len0 + 1 > Lo.cap0) return false;
+  }
+  return true;
+}
+
 int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                           void* stream) {
   if (c && timed_out(c)) return BALANCEKV_E_TIMEOUT;
@@ -878,7 +903,8 @@ int balancekv_stream_step(balancekv_ctx* c, int layer, const void* q, const void
       const int early = alike && c->decode_chain && c->chain_stream == st;
       ProfScope ps(c, 4, st);
       BKV_CUDA(launch_decode_step_mma(c->G, c->A, layer, q, out, c->d_decode_scratch, splits, c->d_status, c->decode_maps,
-                                      k_new, v_new, rel, idx0, new_len, alike ? hint : nullptr, early, st));
+                                      k_new, v_new, rel, idx0, new_len, alike ? hint : nullptr, early, c->step_flag, c->step_expect, st));
+      c->step_flag = nullptr;
       c->decode_chain = true;
       c->chain_stream = st;
       c->kernels_launched++;
@@ -896,32 +922,65 @@ int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)c->cfg.n_seqs * c->cfg.n_q_heads * c->cfg.head_dim * c->esz;
   const size_t kb = (size_t)c->cfg.n_seqs * c->cfg.n_kv_heads * c->cfg.head_dim * c->esz;
+  const size_t payload = (qb + 2 * kb + 15) / 16 * 16;
   if (!c->step_host) {   // first call: staging buffers (allocates)
-    c->step_slot_bytes = (qb + 2 * kb + 255) / 256 * 256;
+    c->step_slot_bytes = (payload + 16 + 255) / 256 * 256;          // q | k | v | arrival flag
     BKV_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->step_host), c->step_slot_bytes * balancekv_ctx::kStepSlots,
                            cudaHostAllocDefault));
+    std::memset(c->step_host, 0, c->step_slot_bytes * balancekv_ctx::kStepSlots);
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->step_dev_in), c->step_slot_bytes * balancekv_ctx::kStepSlots));
+    BKV_CUDA(cudaMemset(c->step_dev_in, 0, c->step_slot_bytes * balancekv_ctx::kStepSlots));
     BKV_CUDA(cudaMalloc(&c->step_dev_out, qb));
     c->bytes_resident += c->step_slot_bytes * balancekv_ctx::kStepSlots + qb;
     for (cudaEvent_t& e : c->step_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     for (cudaEvent_t& e : c->step_used_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-    BKV_CUDA(cudaStreamCreateWithFlags(&c->step_copy_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& e : c->step_group_ev) BKV_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    if (!c->step_copy_stream) BKV_CUDA(cudaStreamCreateWithFlags(&c->step_copy_stream, cudaStreamNonBlocking));
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      c->write_value_fn = fn;
+    else
+      (void)cudaGetLastError();
   }
   // The three small inputs travel as one copy: packed into a pinned slot on the host, then one
   // host-to-device transfer into the slot's device twin on the library's copy stream, so that the
-  // transfer of a step runs while the previous step's kernel does; the kernel waits for its
-  // transfer through an event.  A slot pair is reused only after the kernel that read it has finished.
-  const int slot = (int)(c->step_count % balancekv_ctx::kStepSlots);
-  if (c->step_count >= (unsigned long long)balancekv_ctx::kStepSlots) BKV_CUDA(cudaEventSynchronize(c->step_used_ev[slot]));
-  ++c->step_count;
+  // transfer of a step runs while the previous step's kernel does.  With the fused step kernel no event
+  // ties the launch to the transfer (an event wait between two steps would keep the next step's CTAs
+  // from becoming resident early): a second small copy writes an arrival word behind the operands and
+  // the kernel waits, bounded, for that word.  Otherwise the step's kernels wait for the transfer
+  // through an event.  A slot is reused only after the kernel that read it has finished (one event
+  // per 16 steps).
+  constexpr int kSlots = balancekv_ctx::kStepSlots, kGroup = kSlots / 4;
+  const unsigned long long n = c->step_count++;
+  const int slot = (int)(n % kSlots), group = slot / kGroup;
+  if (n >= (unsigned long long)kSlots && slot % kGroup == 0) BKV_CUDA(cudaEventSynchronize(c->step_group_ev[group]));
   char* h = c->step_host + (size_t)slot * c->step_slot_bytes;
   char* dev_in = c->step_dev_in + (size_t)slot * c->step_slot_bytes;
   std::memcpy(h, q_host, qb);
   std::memcpy(h + qb, k_host, kb);
   std::memcpy(h + qb + kb, v_host, kb);
+  const bool fused = step_can_fuse(c, layer);
   BKV_CUDA(cudaMemcpyAsync(dev_in, h, qb + 2 * kb, cudaMemcpyHostToDevice, c->step_copy_stream));
-  BKV_CUDA(cudaEventRecord(c->step_ev[slot], c->step_copy_stream));
-  BKV_CUDA(cudaStreamWaitEvent(st, c->step_ev[slot], 0));
+  if (fused) {
+    const int expect = (int)((n + 1) & 0x7fffffffu);
+    // the arrival word: a stream memory operation behind the transfer (a 16-byte copy where the driver has none)
+    typedef CUresult (*WriteValueFn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+    bool written = false;
+    if (c->write_value_fn)
+      written = reinterpret_cast<WriteValueFn>(c->write_value_fn)(c->step_copy_stream, (CUdeviceptr)(uintptr_t)(dev_in + payload),
+                                                                  (cuuint32_t)expect, 0) == CUDA_SUCCESS;
+    if (!written) {
+      *reinterpret_cast<int*>(h + payload) = expect;
+      BKV_CUDA(cudaMemcpyAsync(dev_in + payload, h + payload, 16, cudaMemcpyHostToDevice, c->step_copy_stream));
+    }
+    c->step_flag = reinterpret_cast<const int*>(dev_in + payload);
+    c->step_expect = expect;
+  } else {
+    BKV_CUDA(cudaEventRecord(c->step_ev[slot], c->step_copy_stream));
+    BKV_CUDA(cudaStreamWaitEvent(st, c->step_ev[slot], 0));
+  }
   // A pinned (mapped) result buffer is written by the kernel itself: the 8 KB of a step then need
   // no transfer of their own.  Pageable memory goes through the device buffer and a copy.
   void* out_dev = nullptr;
@@ -934,7 +993,8 @@ int balancekv_stream_step_host(balancekv_ctx* c, int layer, const void* q_host, 
       (void)cudaGetLastError();
   }
   int rc = balancekv_stream_step(c, layer, dev_in, dev_in + qb, dev_in + qb + kb, out_dev ? out_dev : c->step_dev_out, stream);
-  BKV_CUDA(cudaEventRecord(c->step_used_ev[slot], st));
+  c->step_flag = nullptr;
+  if (slot % kGroup == kGroup - 1) BKV_CUDA(cudaEventRecord(c->step_group_ev[group], st));
   if (rc) return rc;
   if (!out_dev) BKV_CUDA(cudaMemcpyAsync(out_host, c->step_dev_out, qb, cudaMemcpyDeviceToHost, st));
   return BALANCEKV_OK;

@@ -149,6 +149,12 @@ struct StepAppend {
   // appended.  Every other tile may then be fetched before the grid dependency is resolved (see
   // the kernel's prologue).  Needs the segment table as a parameter (n_seg > 0).
   int early;
+  // The step's operands (q, k_new, v_new) arrive by a copy on another CUDA stream that no event ties to
+  // this launch: the copy is followed by a copy of the word `in_expect` to *in_flag, and the kernel
+  // waits (bounded) for that word before it reads them.  nullptr: the operands are ordered before the
+  // launch in the usual way.
+  const int* in_flag;
+  int in_expect;
 };
 
 struct TileRef {
@@ -239,7 +245,9 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   // The step's operands are wanted right after the dependency resolves: ask for them in L2 now.  A
   // line fetched before its producer has written it is harmless, L2 being the point of coherence
   // (the producer's write updates that line; nothing is taken into L1 here).
-  if (tid < 2 * g) {
+  if (ap.in_flag) {
+    // operands still in flight: nothing to ask for yet
+  } else if (tid < 2 * g) {
     const char* qrow = reinterpret_cast<const char*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + (tid >> 1)) * kD);
     asm volatile("prefetch.global.L2 [%0];" ::"l"(qrow + 128 * (tid & 1)));
   } else if (ap.k_new && tid < 2 * g + 4) {
@@ -286,6 +294,17 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0)
       while (issued < min(kStages, my_tiles)) issue(issued++);
+  }
+  if (ap.in_flag) {
+    // the copy engine writes the operands, then the flag word (two copies in stream order)
+    if (tid == 0) {
+      const long long t0 = clock64();
+      while (*reinterpret_cast<const volatile int*>(ap.in_flag) != ap.in_expect) {
+        if (clock64() - t0 > kWaitCycles) { atomicCAS(status, kStatusOk, kStatusWaitTimeout); break; }
+      }
+      __threadfence();
+    }
+    __syncthreads();
   }
 
   // B fragments of the query tile (k = dims, n = query head of the group; heads >= g are zero).
@@ -775,7 +794,8 @@ void decode_mma_release(void* maps) { delete static_cast<DecodeMaps*>(maps); }
 
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st);
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, const int* in_flag,
+                                   int in_expect, cudaStream_t st);
 
 // Scratch layout of all launches: ticket counters, then (stream, split, head) rows of kD column sums,
 // then their (max, sum) pairs.
@@ -789,7 +809,7 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u, 0};
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
                                                         tickets, status, ap, tm->k, tm->v);
   return cudaGetLastError();
@@ -807,7 +827,7 @@ cudaError_t launch_decode_parts_mma_slots(const Geom& G, const Arena& A, const i
   unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits, n_slots);
-  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words, 0};
+  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words, 0, nullptr, 0};
   for (int i = 0; i < n_slots; ++i) ap.slot_layer[i] = slot_layers[i];
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, slot_layers[0], static_cast<const __nv_bfloat16*>(q), nullptr,
                                                         part, tickets, status, ap, tm->k, tm->v);
@@ -852,7 +872,8 @@ cudaError_t launch_merged_ratio(const float* acc, const float* ml, int n_parts, 
 // [B*H, d] bf16; all streams of the layer have the same level-0 fill).  k_new == nullptr: plain decode.
 cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,
                                    int splits, int* status, const void* maps, const void* k_new, const void* v_new,
-                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, cudaStream_t st) {
+                                   int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, const int* in_flag,
+                                   int in_expect, cudaStream_t st) {
   if (!maps) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
@@ -860,12 +881,14 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   float* part = scratch + ((n_sl + 63) / 64) * 64;
   dim3 grid(n_sl, splits);
   StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u, 0};
+                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0};
   if (seg_hint) {
     ap.n_seg = G.T + 1;
     for (int l = 0; l <= G.T; ++l) ap.seg[l] = seg_hint[l];
     ap.early = early ? 1 : 0;
   }
+  ap.in_flag = in_flag;
+  ap.in_expect = in_expect;
   // programmatic stream serialization: back-to-back decode steps overlap a launch with the
   // previous kernel's tail (see the kernel's prologue)
   cudaLaunchConfig_t cfg = {};
