@@ -51,6 +51,16 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
     }                                                                                     \
   } while (0)
 
+// Split-K scratch of the decode kernels: ticket counters (CUDA-core kernel: zero, self-resetting), then
+// the partial rows.  The tensor-core kernel uses a word of a partial row as its own arrival flag: between
+// launches every such word holds the all-ones pattern, which the combining CTA restores after reading.
+static cudaError_t init_decode_scratch(float* scratch, size_t bytes, size_t n_sl, cudaStream_t st) {
+  const size_t ticket_bytes = ((n_sl + 63) / 64) * 64 * sizeof(unsigned);
+  cudaError_t e = cudaMemsetAsync(scratch, 0xff, bytes, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(scratch, 0, ticket_bytes < bytes ? ticket_bytes : bytes, st);
+  return e;
+}
+
 struct balancekv_ctx {
   balancekv_config cfg{};
   Geom G{};
@@ -363,7 +373,8 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
     if (f.decode_splits > 0) c->max_splits = std::min(64, f.decode_splits);
     const size_t sb = decode_scratch_bytes(G, c->max_splits);
     if ((rc = dev_alloc(c, reinterpret_cast<char**>(&c->d_decode_scratch), sb))) return fail(rc);
-    if (cudaMemset(c->d_decode_scratch, 0, sb) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+    if (init_decode_scratch(c->d_decode_scratch, sb, (size_t)G.B * G.H, nullptr) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
+    if (cudaStreamSynchronize(nullptr) != cudaSuccess) return fail(BALANCEKV_E_CUDA);
   }
   c->ring_half = (size_t)4 << 20;
   if (cudaMallocHost(reinterpret_cast<void**>(&c->h_ring), 2 * c->ring_half) != cudaSuccess) return fail(BALANCEKV_E_NOMEM);
@@ -707,6 +718,14 @@ static bool layer_seg_hint(balancekv_ctx* c, int layer, Seg* out) {
 }
 
 // Split-K factor of a decode launch over the layer's current caches.
+// The tensor-core decode kernel adds g - 1 combining CTAs per stream to a launch with more than one split:
+// the largest split factor <= splits whose grid over n_streams streams still fits one wave.
+static int one_wave_splits(balancekv_ctx* c, int splits, int n_streams) {
+  const int per_stream = c->decode_slots / std::max(1, n_streams);
+  const int room = per_stream - (c->cfg.n_q_heads / c->cfg.n_kv_heads - 1);
+  return std::max(1, std::min(splits, room));
+}
+
 static int pick_splits(balancekv_ctx* c, int layer) {
   const balancekv_config& f = c->cfg;
   int64_t max_rows = 0;
@@ -723,6 +742,7 @@ static int pick_splits(balancekv_ctx* c, int layer) {
   // the fewest splits with the same number of tiles per CTA: the tile phase is as long, the combine shorter
   const int64_t tiles_per = std::max<int64_t>(1, (tiles + splits - 1) / splits);
   splits = (int)std::max<int64_t>(1, (tiles + tiles_per - 1) / tiles_per);
+  if (c->decode_maps) splits = one_wave_splits(c, splits, c->cfg.n_seqs * c->cfg.n_kv_heads);
   if (f.decode_splits > 0) splits = std::min(f.decode_splits, c->max_splits);
   return splits;
 }
@@ -824,10 +844,12 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_acc), sizeof(float) * (size_t)n_heads * d * BALANCEKV_MAX_MERGE));
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_ml), sizeof(float) * (size_t)n_heads * 2 * BALANCEKV_MAX_MERGE));
     c->bytes_resident += sizeof(float) * (size_t)n_heads * (d + 2) * BALANCEKV_MAX_MERGE;
-    // one split-K scratch block per slot, so that all slots go in one launch; tickets start at zero
+    // one split-K scratch block per slot, so that all slots go in one launch
     const size_t block_bytes = (decode_scratch_bytes(c->G, c->max_splits) + 255) & ~(size_t)255;
     BKV_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->two_scratch), block_bytes * BALANCEKV_MAX_MERGE));
-    BKV_CUDA(cudaMemsetAsync(c->two_scratch, 0, block_bytes * BALANCEKV_MAX_MERGE, st));
+    for (int z = 0; z < BALANCEKV_MAX_MERGE; ++z)
+      BKV_CUDA(init_decode_scratch(reinterpret_cast<float*>(reinterpret_cast<char*>(c->two_scratch) + block_bytes * z), block_bytes,
+                                   (size_t)c->G.B * c->G.H, st));
     c->two_scratch_words = block_bytes / 4;
     c->bytes_resident += block_bytes * BALANCEKV_MAX_MERGE;
   }
@@ -840,7 +862,7 @@ int balancekv_decode_attn_merged(balancekv_ctx* c, const int32_t* layers_num, in
     if (!((num_mask >> p) & 1u)) keys_mask |= 1u << p;     // a slot that only enters the denominator: values are not read
   }
   const int n_sl = c->cfg.n_seqs * c->cfg.n_kv_heads;
-  splits = std::max(1, std::min(splits, c->decode_slots / std::max(1, n_sl * n_parts)));
+  splits = one_wave_splits(c, splits, n_sl * n_parts);
   {
     ProfScope ps(c, 4, st);
     BKV_CUDA(launch_decode_parts_mma_slots(c->G, c->A, slots, n_parts, keys_mask, q, c->two_acc, c->two_ml, c->two_scratch,
@@ -1272,6 +1294,11 @@ int balancekv_reset(balancekv_ctx* c, void* stream) {
   // a context that gave up on a device-side wait becomes usable again
   BKV_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(int), st));
   *c->h_status = 0;
+  // a launch that gave up may have left partial rows behind
+  BKV_CUDA(init_decode_scratch(c->d_decode_scratch, decode_scratch_bytes(c->G, c->max_splits), (size_t)c->G.B * c->G.H, st));
+  if (c->two_scratch)
+    for (int z = 0; z < BALANCEKV_MAX_MERGE; ++z)
+      BKV_CUDA(init_decode_scratch(c->two_scratch + c->two_scratch_words * z, c->two_scratch_words * 4, (size_t)c->G.B * c->G.H, st));
   return BALANCEKV_OK;
 }
 

@@ -48,7 +48,6 @@ constexpr uint32_t kHalf = kTN * 128;        // bytes of one [64 tokens][64 dims
 constexpr uint32_t kTensorBytes = 2 * kHalf; // K (or V) tile: two boxes
 constexpr uint32_t kStageBytes = 2 * kTensorBytes;
 constexpr long long kWaitCycles = 100000000LL;   // about 50 ms: a bulk copy that has not landed by then never will
-constexpr int kChunks = 1;                   // barriers of the combine's staging copy
 constexpr int PS = kD + 4;                   // row of the in-CTA merge buffer: acc[D], max, sum, 2 pad (bank-conflict free)
 
 struct DecodeMaps {
@@ -110,6 +109,20 @@ __device__ inline float fast_exp2(float x) {     // -inf -> 0
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Polling loads of the split-K scratch (see the combine): never served by L1.
+constexpr uint32_t kEmptyWord = 0xffffffffu;
+constexpr int kMaxSplits = 64;
+__device__ inline bool is_empty(float x) { return __float_as_uint(x) == kEmptyWord; }
+__device__ inline float ld_poll1(const float* p) {
+  float v;
+  asm volatile("ld.volatile.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ inline float2 ld_poll2(const float* p) {
+  float2 v;
+  asm volatile("ld.volatile.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+  return v;
+}
 __device__ inline uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -138,7 +151,7 @@ struct StepAppend {
   Seg seg[kMaxLevels + 1];
   // One launch over several layer slots (decode merged over slots): blockIdx.z selects the slot.
   // n_slots = 0: a launch over the one slot `layer`.  z_stride: 4-byte words between the scratch
-  // blocks (tickets, partial rows) of consecutive slots; raw_acc / raw_ml advance by one
+  // blocks (partial rows and their pairs) of consecutive slots; raw_acc / raw_ml advance by one
   // [B, H g, d] / [B, H g, 2] block per slot; bit z of keys_mask = keys_only of slot z.
   int n_slots;
   int slot_layer[8];
@@ -155,6 +168,9 @@ struct StepAppend {
   // launch in the usual way.
   const int* in_flag;
   int in_expect;
+  // Splits of a stream's tiles.  With more than one the grid has g - 1 more CTAs per stream, which combine
+  // the heads 1 .. g - 1 (see the kernel's combine).
+  int splits;
 };
 
 struct TileRef {
@@ -192,10 +208,9 @@ __device__ inline bool group_bar_or(int group, bool pred) {
 
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
-                  float* __restrict__ part_base, unsigned* __restrict__ tickets_base, int* __restrict__ status,
+                  float* __restrict__ part_base, int* __restrict__ status,
                   const StepAppend ap, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
   float* part = part_base;
-  unsigned* tickets = tickets_base;
   float* raw_acc = ap.raw_acc;
   float* raw_ml = ap.raw_ml;
   int keys_only = ap.keys_only;
@@ -204,7 +219,6 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     layer = ap.slot_layer[z];
     keys_only = (int)((ap.keys_mask >> z) & 1u);
     part += (size_t)z * ap.z_stride;
-    tickets += (size_t)z * ap.z_stride;
     raw_acc += (size_t)z * G.B * G.H * G.g * kD;
     raw_ml += (size_t)z * G.B * G.H * G.g * 2;
   }
@@ -213,7 +227,6 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   uint64_t* full = reinterpret_cast<uint64_t*>(tiles + kStages * kStageBytes);
   __shared__ int lvl_tiles[kMaxLevels + 1];
   __shared__ Seg seg_s[kMaxLevels + 1];
-  __shared__ int is_last_s;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int group = warp / kGroupWarps, wq = warp % kGroupWarps;   // tile parity served, token quarter of the tile
@@ -221,7 +234,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const int sl = blockIdx.x;
   const int seq = sl / G.H, head = sl % G.H;
   const int stream = (seq * G.L + layer) * G.H + head;
-  const int splits = gridDim.y, split = blockIdx.y;
+  const int splits = ap.splits, split = blockIdx.y;     // split >= splits: a combiner without tiles (see the combine)
   const int64_t stream_base = (int64_t)stream * G.rows_per_stream;
   // Merge and combine phases: the first work item of this warp, (head mh, way mw) with warp = mw g + mh.
   int mh = warp, mw = 0;
@@ -236,7 +249,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   // one earlier launch of the chain is ever in flight.  Without the launch attribute both
   // instructions do nothing.
   if (tid == 0) {
-    for (int s = 0; s < kBars + kChunks; ++s) mbar_init(&full[s], 1);     // full[kBars ..]: the combine's staging copies
+    for (int s = 0; s < kBars; ++s) mbar_init(&full[s], 1);
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmK) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmV) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -270,7 +283,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   for (int l = 0; l <= G.T; ++l) n_tiles += lvl_tiles[l];
   const int t_begin = (int)((long long)n_tiles * split / splits);
   const int t_end = (int)((long long)n_tiles * (split + 1) / splits);
-  const int my_tiles = t_end - t_begin;
+  const int my_tiles = split < splits ? t_end - t_begin : 0;
 
   auto issue = [&](int i) {   // one thread
     const TileRef tr = locate_tile(t_begin + i, lvl_tiles, seg_s, G.T, stream_base, G.region_off);
@@ -307,6 +320,151 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     __syncthreads();
   }
 
+  const float sc = 1.4426950408889634f * G.inv_sqrt_d;
+
+  // ---- the end of a head's path, by all threads of a CTA (thread = output column): the appended token
+  // joins as one more partial (level 0, weight 1, <q, k_new> in fp32), the ratio or the raw parts are
+  // written, and with h == 0 the token's row goes into the cache.
+  struct NewTok {
+    uint2 kn;                  // 4 dims of k_new per lane
+    uint2 qv[kMaxGroup];       // 4 dims of q per lane and head (one head: slot 0)
+    float vn;                  // column tid of v_new
+    uint4 row_new;             // last warp: lanes 0-15 a piece of the row of K, lanes 16-31 of V
+  };
+  // h < 0: the queries of all heads
+  auto load_new = [&](int h) -> NewTok {
+    NewTok nt;
+    nt.kn = make_uint2(0u, 0u);
+    nt.vn = 0.f;
+    nt.row_new = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int k = 0; k < kMaxGroup; ++k) nt.qv[k] = make_uint2(0u, 0u);
+    if (ap.k_new) {
+      nt.kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
+      nt.vn = __bfloat162float(ap.v_new[(size_t)sl * kD + tid]);
+      const __nv_bfloat16* qs = q + ((size_t)seq * (G.H * g) + (size_t)head * g) * kD + 4 * lane;
+      if (h >= 0) {
+        nt.qv[0] = *reinterpret_cast<const uint2*>(qs + (size_t)h * kD);
+      } else {
+#pragma unroll
+        for (int k = 0; k < kMaxGroup; ++k)
+          if (k < g) nt.qv[k] = *reinterpret_cast<const uint2*>(qs + (size_t)k * kD);
+      }
+      if (h <= 0 && warp == kWarps - 1)
+        nt.row_new = reinterpret_cast<const uint4*>((lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD)[lane & 15];
+    }
+    return nt;
+  };
+  auto finish = [&](int h, float a, float M, float L, const NewTok& nt, int qslot) {
+    if (ap.k_new) {
+      const uint2 qv = nt.qv[qslot];
+      const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.y);
+      const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv.y);
+      float dot = __bfloat162float(q01.x) * __bfloat162float(k01.x);
+      dot = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), dot);
+      dot = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), dot);
+      dot = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), dot);
+      const float x = warp_sum(dot) * sc;
+      const float Mn = fmaxf(M, x);
+      const float f = M == -INFINITY ? 0.f : fast_exp2(M - Mn), fN = fast_exp2(x - Mn);
+      a = fmaf(nt.vn, fN, a * f);
+      L = fmaf(L, f, fN);
+      M = Mn;
+    }
+    const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
+    if (raw_acc) {
+      raw_acc[qh * kD + tid] = a;
+      if (tid == 0) { raw_ml[2 * qh] = M; raw_ml[2 * qh + 1] = L; }
+    } else {
+      const float inv = L > 0.f ? 1.0f / L : 0.f;
+      out[qh * kD + tid] = __float2bfloat16_rn(a * inv);
+    }
+    if (ap.k_new && h == 0 && warp == kWarps - 1) {
+      // append: one 256-byte row of K and of V, the position, the new length of C^0
+      const size_t dst_row = (size_t)stream_base + G.region_off[0] + ap.rel_row;
+      __nv_bfloat16* dstp = static_cast<__nv_bfloat16*>(lane < 16 ? A.K : A.V) + dst_row * kD;
+      reinterpret_cast<uint4*>(dstp)[lane & 15] = nt.row_new;
+      float s2 = 0.f;                                         // ||k||^2 / ||v||^2 travel with the row
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&nt.row_new);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 fv = __bfloat1622float2(h2[i]);
+        s2 = fmaf(fv.x, fv.x, s2);
+        s2 = fmaf(fv.y, fv.y, s2);
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+      const float v2 = __shfl_sync(0xffffffffu, s2, 16);
+      if (lane == 0 && A.nrm) A.nrm[dst_row] = make_float2(s2, v2);
+      if (lane == 1) {
+        A.idx[dst_row] = ap.idx0;
+        A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
+      }
+    }
+  };
+  // Combine head h of this CTA's stream (all threads; thread = output column; see the combine below).
+  auto combine_head = [&](int h) {
+    const float* rows = part + ((size_t)sl * splits * g + h) * kD + tid;                         // row of split sp: + sp rstep
+    const float* mls = part + (size_t)gridDim.x * splits * g * kD + ((size_t)sl * splits * g + h) * 2;   // its pair: + sp g 2
+    const size_t rstep = (size_t)g * kD;
+    const NewTok nt = load_new(h);              // in flight during the polls
+    const float* mlp[2] = {mls + (size_t)lane * g * 2, mls + (size_t)(lane + 32) * g * 2};
+    float2 ml[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) ml[e] = lane + 32 * e < splits ? ld_poll2(mlp[e]) : make_float2(-INFINITY, 0.f);
+    float v[kMaxSplits];
+#pragma unroll
+    for (int j = 0; j < kMaxSplits; ++j)
+      if (j < splits) v[j] = ld_poll1(rows + j * rstep);
+    // A round re-reads everything that was still empty, all loads in flight together (words checked one
+    // after the other would cost a round trip each).
+    const long long t0 = clock64();
+    bool ok = true;
+    for (;;) {
+      bool pending = false;
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+        if (lane + 32 * e < splits && (is_empty(ml[e].x) || is_empty(ml[e].y))) {
+          ml[e] = ld_poll2(mlp[e]);
+          pending = true;
+        }
+#pragma unroll
+      for (int j = 0; j < kMaxSplits; ++j)
+        if (j < splits && is_empty(v[j])) {
+          v[j] = ld_poll1(rows + j * rstep);
+          pending = true;
+        }
+      if (!pending) break;
+      if (clock64() - t0 > kWaitCycles) { ok = false; break; }
+    }
+    __syncwarp();
+    const float M = warp_max(fmaxf(ml[0].x, ml[1].x));
+    const float f0 = ml[0].x == -INFINITY ? 0.f : fast_exp2(ml[0].x - M);
+    const float f1 = ml[1].x == -INFINITY ? 0.f : fast_exp2(ml[1].x - M);
+    const float L = warp_sum(fmaf(ml[0].y, f0, ml[1].y * f1));
+    float a = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxSplits; ++j)
+      if (j < splits) a = fmaf(v[j], __shfl_sync(0xffffffffu, j < 32 ? f0 : f1, j & 31), a);
+    finish(h, a, M, L, nt, 0);
+    // the empty pattern again, for the next launch (the pairs once every warp has read them)
+    const float e = __uint_as_float(kEmptyWord);
+#pragma unroll
+    for (int j = 0; j < kMaxSplits; ++j)
+      if (j < splits) __stcg(const_cast<float*>(rows + j * rstep), e);
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+      for (int k = 0; k < 2; ++k)
+        if (lane + 32 * k < splits) __stcg(reinterpret_cast<float2*>(const_cast<float*>(mlp[k])), make_float2(e, e));
+    }
+    if (!ok && lane == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
+  };
+  if (split >= splits) {                        // a CTA without tiles: the combiner of head split - splits + 1
+    combine_head(split - splits + 1);
+    return;
+  }
+
   // B fragments of the query tile (k = dims, n = query head of the group; heads >= g are zero).
   // The tokens are the M dimension of both products (S^T = K Q^T, O^T = V^T P^T), so a warp spends
   // one mma.sync.m16n8k16 per 16 tokens x 16 dims instead of the two that a query-major tile
@@ -325,7 +483,6 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       qb[ks][0] = lo; qb[ks][1] = hi;
     }
   }
-  const float sc = 1.4426950408889634f * G.inv_sqrt_d;
 
   // O^T of this warp's tokens: o[mb][j] = dim 16 mb + hq + 8 (j >> 1), query head 2 tq + (j & 1)
   float o[8][4];
@@ -528,238 +685,51 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y); acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
         L = fmaf(rowp[kD + 1], f, L);
       }
-      *reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane) = acc;
-      if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
-    }
-  }
-  // ---- ticket: the last CTA of the stream combines the splits
-  if (!single) {
-    // release / acquire through one thread: the barrier orders the CTA's writes before thread 0's
-    // fence and its fence after the ticket before everybody's reads (fences are cumulative); a
-    // fence by every thread costs a microsecond here
-    __syncthreads();
-    if (tid == 0) {
-      __threadfence();
-      const unsigned old = atomicAdd(&tickets[sl], 1u);
-      is_last_s = old == (unsigned)(splits - 1);
-      if (is_last_s) __threadfence();
-    }
-    __syncthreads();
-    if (!is_last_s) return;
-  } else {
-    __syncthreads();
-  }
-  // Combine.  All partial rows of the stream are contiguous; if they fit, one bulk copy brings them
-  // into the idle tile ring, otherwise they are read from global memory.  The (max, sum) pairs of
-  // all splits are read straight from L2 meanwhile and turned into the scale factors of the splits.
-  // Every global load of this phase is issued before the first of them is consumed: the CTA is
-  // alone on the critical path here, and each dependent round trip would show.
-  const float* sp = part + (size_t)sl * splits * g * kD;
-  const float* sp_ml = single ? my_ml : part + n_rows_all * kD + (size_t)sl * splits * g * 2;
-  float* cm = reinterpret_cast<float*>(tiles);            // [splits][g] max, later the scale factors
-  float* cl = cm + 64 * kMaxGroup;                        // [splits][g] sums
-  float* cM = cl + 64 * kMaxGroup;                        // [g] overall max
-  float* cL = cM + kMaxGroup;                             // [g] overall sum
-  float* cN = cL + kMaxGroup;                             // [g] factor of the appended token
-  constexpr uint32_t kStageOff = 4352 + kWarps * kMaxGroup * 32 * 16;   // behind cm, cl, cM, cL, cN and the column-sum parts
-  const uint32_t part_bytes = (uint32_t)splits * g * kD * sizeof(float);
-  const bool staged = single || part_bytes <= kStages * kStageBytes - kStageOff;
-  const float* sp_s = reinterpret_cast<const float*>(tiles + (single ? kSingleOff : kStageOff));
-  uint64_t* cbar = full + kBars;
-  if (staged && !single && tid == kThreads - 32) {
-    // earlier generic-proxy accesses to this shared memory and the other CTAs' global writes
-    // (acquired above) come before the async-proxy copy
-    asm volatile("fence.proxy.async;" ::: "memory");
-    mbar_expect_tx(cbar, part_bytes);
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(tiles + kStageOff)), "l"(sp), "r"(part_bytes), "r"(smem_u32(cbar)) : "memory");
-  }
-  // ---- loads: (max, sum) pairs; the appended token's rows (last warp) and, per lane, 4 dims of k_new
-  // and of q and 4 columns of v_new for this warp's heads
-  constexpr int kMlPer = (64 * kMaxGroup + kThreads - 1) / kThreads;
-  constexpr int kHeadsPer = (kMaxGroup + kWarps - 1) / kWarps;
-  float2 mlv[kMlPer];
-#pragma unroll
-  for (int k = 0; k < kMlPer; ++k) {
-    const int i = tid + k * kThreads;
-    mlv[k] = make_float2(-INFINITY, 0.f);
-    if (i < splits * g) {
-      const float2* mlp = reinterpret_cast<const float2*>(sp_ml) + i;
-      mlv[k] = single ? *mlp : __ldcg(mlp);
-    }
-  }
-  const size_t dst_row = (size_t)stream_base + G.region_off[0] + ap.rel_row;
-  uint4 row_new = make_uint4(0u, 0u, 0u, 0u);
-  uint2 kn = make_uint2(0u, 0u), qv[kHeadsPer], vn_pre = make_uint2(0u, 0u);
-  if (ap.k_new) {
-    if (warp == kWarps - 1)                                   // lanes 0-15: the row of K, lanes 16-31: the row of V
-      row_new = reinterpret_cast<const uint4*>((lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD)[lane & 15];
-    if (warp < g) {
-      kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
-      vn_pre = *reinterpret_cast<const uint2*>(ap.v_new + (size_t)sl * kD + 4 * lane);
-#pragma unroll
-      for (int k = 0; k < kHeadsPer; ++k) {
-        const int h = warp + k * kWarps;
-        qv[k] = h < g ? *reinterpret_cast<const uint2*>(q + ((size_t)seq * (G.H * g) + (size_t)head * g + h) * kD + 4 * lane)
-                      : make_uint2(0u, 0u);
+      if (single) {
+        *reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane) = acc;
+        if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
+      } else {                                  // published: see the combine below
+        __stcg(reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane), acc);
+        if (lane == 0) __stcg(reinterpret_cast<float2*>(my_ml + 2 * h), make_float2(M, L));
       }
     }
   }
-  // ---- consume
+  // ---- combine.  No ticket, no fence and no staging copy: a word of the scratch is its own arrival flag.
+  // Between launches every word of the partial rows holds kEmptyWord, a NaN pattern that arithmetic never
+  // produces (results are canonical NaNs, and -inf is a legal maximum).  A CTA publishes its rows with plain
+  // stores.  Head 0 of a stream is combined by the stream's CTA of the last split, head h > 0 by the CTA
+  // (stream, splits + h - 1), which has no tiles: the g combiners of a stream run side by side on different
+  // SMs, each polls the words of its head until none is empty, sums, and puts the empty pattern back for the
+  // next launch.  CTAs are dispatched in index order, so everything a combiner waits for was dispatched
+  // before it and never waits itself: the wait ends (and is bounded anyway).  The chain behind the last tile
+  // is then one store and about one load through L2 instead of fence, ticket, fence and copy.
+  if (single) {
+    __syncthreads();                            // the rows in shared memory are complete
+    const float* acc1 = reinterpret_cast<const float*>(tiles + kSingleOff);
+    const float* ml1 = acc1 + kMaxGroup * kD;
+    NewTok nt = load_new(-1);
 #pragma unroll
-  for (int k = 0; k < kMlPer; ++k) {
-    const int i = tid + k * kThreads;
-    if (i < splits * g) { cm[i] = mlv[k].x; cl[i] = mlv[k].y; }
+    for (int h = 0; h < kMaxGroup; ++h)
+      if (h < g) finish(h, acc1[h * kD + tid], ml1[2 * h], ml1[2 * h + 1], nt, h);
+    return;
   }
-  float x_new[kHeadsPer];
-#pragma unroll
-  for (int k = 0; k < kHeadsPer; ++k) x_new[k] = 0.f;
-  if (ap.k_new) {
-    // append (every CTA of the stream has taken its ticket, so nobody reads the old segment table
-    // any more): one 256-byte row of K and of V, the position, the new length of C^0.
-    if (warp == kWarps - 1) {
-      __nv_bfloat16* dstp = static_cast<__nv_bfloat16*>(lane < 16 ? A.K : A.V) + dst_row * kD;
-      reinterpret_cast<uint4*>(dstp)[lane & 15] = row_new;
-      float s2 = 0.f;                                         // ||k||^2 / ||v||^2 travel with the row
-      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&row_new);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __bfloat1622float2(h2[i]);
-        s2 = fmaf(f.x, f.x, s2);
-        s2 = fmaf(f.y, f.y, s2);
-      }
-#pragma unroll
-      for (int o = 8; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-      const float v2 = __shfl_sync(0xffffffffu, s2, 16);
-      if (lane == 0 && A.nrm) A.nrm[dst_row] = make_float2(s2, v2);
-      if (lane == 1) {
-        A.idx[dst_row] = ap.idx0;
-        A.seg[(size_t)stream * (G.T + 1)].len = ap.new_len;
-      }
-    }
-    if (warp < g) {
-      // the appended token: level 0, weight 1; <q, k_new> in fp32, 4 dims per lane
-      const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&kn.y);
-#pragma unroll
-      for (int k = 0; k < kHeadsPer; ++k) {
-        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv[k].x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv[k].y);
-        float dot = __bfloat162float(q01.x) * __bfloat162float(k01.x);
-        dot = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), dot);
-        dot = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), dot);
-        dot = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), dot);
-        x_new[k] = warp_sum(dot) * sc;
-      }
-    }
-  }
-  __syncthreads();
-#pragma unroll
-  for (int k = 0; k < kHeadsPer; ++k) {        // one warp per head, lanes over the (<= 64) splits
-    const int h = warp + k * kWarps;
-    if (h >= g) break;
-    const int s0 = lane, s1 = lane + 32;
-    const float m0 = s0 < splits ? cm[s0 * g + h] : -INFINITY, m1 = s1 < splits ? cm[s1 * g + h] : -INFINITY;
-    float M = warp_max(fmaxf(m0, m1));
-    float fN = 0.f;
-    if (ap.k_new) { M = fmaxf(M, x_new[k]); fN = fast_exp2(x_new[k] - M); }
-    const float f0 = m0 == -INFINITY ? 0.f : fast_exp2(m0 - M), f1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - M);
-    float L = (s0 < splits ? cl[s0 * g + h] * f0 : 0.f) + (s1 < splits ? cl[s1 * g + h] * f1 : 0.f);
-    L = warp_sum(L) + fN;
-    if (s0 < splits) cm[s0 * g + h] = f0;
-    if (s1 < splits) cm[s1 * g + h] = f1;
-    if (lane == 0) { cM[h] = M; cL[h] = L; cN[h] = fN; }
-  }
-  __syncthreads();
-  // Column sums over the splits: warp w takes the splits w, w + kWarps, ... for every head (lane = 4
-  // consecutive columns, one accumulator per head: the chain per thread is splits / kWarps long and the
-  // heads' loads are independent); the warps' parts meet in shared memory, where warp h sums head h.
-  float4 acc[kMaxGroup];
-#pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-  bool landed = true;
-  if (staged && !single) {
-    if (lane == 0) landed = mbar_wait(cbar, 0u);
-    landed = __shfl_sync(0xffffffffu, landed, 0);
-    __syncwarp();
-  }
-  {
-    const size_t row_stride = (size_t)g * kD;
-    for (int sp_i = warp; sp_i < splits; sp_i += kWarps) {
-      const float* fac = cm + (size_t)sp_i * g;
-      if (staged) {
-        const float* p = sp_s + (size_t)sp_i * row_stride + 4 * lane;
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h) {
-          if (h < g) {
-            const float4 v = *reinterpret_cast<const float4*>(p + (size_t)h * kD);
-            const float f = fac[h];
-            acc[h].x = fmaf(v.x, f, acc[h].x); acc[h].y = fmaf(v.y, f, acc[h].y);
-            acc[h].z = fmaf(v.z, f, acc[h].z); acc[h].w = fmaf(v.w, f, acc[h].w);
-          }
-        }
-      } else {
-        const float* p = sp + (size_t)sp_i * row_stride + 4 * lane;
-        float4 v[kMaxGroup];
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-          v[h] = h < g ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)h * kD)) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h) {
-          if (h < g) {
-            const float f = fac[h];
-            acc[h].x = fmaf(v[h].x, f, acc[h].x); acc[h].y = fmaf(v[h].y, f, acc[h].y);
-            acc[h].z = fmaf(v[h].z, f, acc[h].z); acc[h].w = fmaf(v[h].w, f, acc[h].w);
-          }
-        }
-      }
-    }
-  }
-  if (!landed && lane == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
-  float4* red = reinterpret_cast<float4*>(tiles + 4352);  // [kWarps][g][32] partial column sums (<= 16 KB; the staged rows lie behind)
-#pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h)
-    if (h < g) red[((size_t)warp * g + h) * 32 + lane] = acc[h];
-  __syncthreads();
-#pragma unroll
-  for (int k = 0; k < kHeadsPer; ++k) {
-    const int h = warp + k * kWarps;
-    if (h >= g) break;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const float4 r = red[((size_t)w * g + h) * 32 + lane];
-      a.x += r.x; a.y += r.y; a.z += r.z; a.w += r.w;
-    }
-    const int c = 4 * lane;
-    if (ap.k_new) {
-      const float fN = cN[h];
-      const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vn_pre.y);
-      a.x = fmaf(__bfloat162float(v01.x), fN, a.x); a.y = fmaf(__bfloat162float(v01.y), fN, a.y);
-      a.z = fmaf(__bfloat162float(v23.x), fN, a.z); a.w = fmaf(__bfloat162float(v23.y), fN, a.w);
-    }
-    const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
-    if (raw_acc) {
-      *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = a;
-      if (c == 0) { raw_ml[2 * qh] = cM[h]; raw_ml[2 * qh + 1] = cL[h]; }
-    } else {
-      const float inv = cL[h] > 0.f ? 1.0f / cL[h] : 0.f;
-      __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out + qh * kD + c);
-      o2[0] = __floats2bfloat162_rn(a.x * inv, a.y * inv);
-      o2[1] = __floats2bfloat162_rn(a.z * inv, a.w * inv);
-    }
-  }
-  if (tid == 0 && !single) tickets[sl] = 0;   // ready for the next launch
+  if (split == splits - 1) combine_head(0);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (kBars + kChunks) * sizeof(uint64_t);
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kBars * sizeof(uint64_t);
 
 }  // namespace
 
 bool decode_mma_supported(const Geom& G) { return G.is_bf16 && G.d == kD && G.g <= 8; }
 int decode_mma_ctas_per_sm() { return kCtasPerSm; }
+
+// CTAs per stream of a launch with `splits` splits: the combiners of the heads 1 .. g - 1 have CTAs of their own.
+int decode_mma_ctas_per_stream(int g, int splits) { return splits > 1 ? splits + g - 1 : 1; }
+static unsigned grid_y(const Geom& G, int splits) { return (unsigned)decode_mma_ctas_per_stream(G.g, splits); }
 
 // Tensor maps over the K and V arenas viewed as [total_rows, 128] bf16, boxes of 64 dims x 64 rows.
 cudaError_t decode_mma_prepare(const Geom& G, const Arena& A, int64_t total_rows, void** maps_out) {
@@ -806,12 +776,11 @@ cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, co
   if (!maps || !raw_acc || !raw_ml) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
-  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
-  dim3 grid(n_sl, splits);
-  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0};
+  dim3 grid(n_sl, grid_y(G, splits));
+  const StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, keys_only, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0, splits};
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, layer, static_cast<const __nv_bfloat16*>(q), nullptr, part,
-                                                        tickets, status, ap, tm->k, tm->v);
+                                                        status, ap, tm->k, tm->v);
   return cudaGetLastError();
 }
 
@@ -824,13 +793,12 @@ cudaError_t launch_decode_parts_mma_slots(const Geom& G, const Arena& A, const i
   if (!maps || !raw_acc || !raw_ml || n_slots < 1 || n_slots > 8 || z_stride_words > 0xffffffffull) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
-  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
-  dim3 grid(n_sl, splits, n_slots);
-  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words, 0, nullptr, 0};
+  dim3 grid(n_sl, grid_y(G, splits), n_slots);
+  StepAppend ap{nullptr, nullptr, 0, 0, 0, raw_acc, raw_ml, 0, 0, {}, n_slots, {}, keys_mask, (unsigned)z_stride_words, 0, nullptr, 0, splits};
   for (int i = 0; i < n_slots; ++i) ap.slot_layer[i] = slot_layers[i];
   decode_mma_kernel<<<grid, kThreads, kSmemBytes, st>>>(G, A, slot_layers[0], static_cast<const __nv_bfloat16*>(q), nullptr,
-                                                        part, tickets, status, ap, tm->k, tm->v);
+                                                        part, status, ap, tm->k, tm->v);
   return cudaGetLastError();
 }
 
@@ -877,11 +845,10 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   if (!maps) return cudaErrorInvalidValue;
   const DecodeMaps* tm = static_cast<const DecodeMaps*>(maps);
   const int n_sl = G.B * G.H;
-  unsigned* tickets = reinterpret_cast<unsigned*>(scratch);
   float* part = scratch + ((n_sl + 63) / 64) * 64;
-  dim3 grid(n_sl, splits);
+  dim3 grid(n_sl, grid_y(G, splits));
   StepAppend ap{static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), rel_row, idx0,
-                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0};
+                new_len, nullptr, nullptr, 0, 0, {}, 0, {}, 0u, 0u, 0, nullptr, 0, splits};
   if (seg_hint) {
     ap.n_seg = G.T + 1;
     for (int l = 0; l <= G.T; ++l) ap.seg[l] = seg_hint[l];
@@ -902,7 +869,7 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, decode_mma_kernel, G, A, layer, static_cast<const __nv_bfloat16*>(q),
-                            static_cast<__nv_bfloat16*>(out), part, tickets, status, ap, tm->k, tm->v);
+                            static_cast<__nv_bfloat16*>(out), part, status, ap, tm->k, tm->v);
 }
 
 }  // namespace bkv
