@@ -364,7 +364,7 @@ cudaError_t launch_g(const Geom& G, const Arena& A, int layer, const void* q, vo
 // then per (stream, split, head) partial rows of D+2 floats.
 size_t decode_scratch_bytes(const Geom& G, int splits) {
   const size_t n_sl = (size_t)G.B * G.H;
-  return sizeof(float) * (((n_sl + 63) / 64) * 64 + n_sl * splits * G.g * (G.d + 4));   // rows of d + 4 floats cover both decode kernels' layouts
+  return sizeof(float) * (((n_sl + 63) / 64) * 64 + n_sl * splits * G.g * (G.d + 8));   // rows of d + 8 floats cover both decode kernels' layouts
 }
 
 cudaError_t launch_decode(const Geom& G, const Arena& A, int layer, const void* q, void* out, float* scratch,

@@ -113,9 +113,21 @@ __device__ inline float fast_exp2(float x) {     // -inf -> 0
 constexpr uint32_t kEmptyWord = 0xffffffffu;
 constexpr int kMaxSplits = 64;
 __device__ inline bool is_empty(float x) { return __float_as_uint(x) == kEmptyWord; }
-__device__ inline float ld_poll1(const float* p) {
-  float v;
-  asm volatile("ld.volatile.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+// Plain loads as volatile asm statements: they keep their place among the polling loads, i.e. they are issued
+// before the polls and not where their values are first used.
+__device__ inline uint2 ld_early_v2(const void* p) {
+  uint2 v;
+  asm volatile("ld.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  return v;
+}
+__device__ inline uint4 ld_early_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ inline float4 ld_poll4(const float* p) {
+  float4 v;
+  asm volatile("ld.volatile.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
   return v;
 }
 __device__ inline float2 ld_poll2(const float* p) {
@@ -321,6 +333,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   }
 
   const float sc = 1.4426950408889634f * G.inv_sqrt_d;
+  constexpr uint32_t kFacOff = 4352 + kWarps * kMaxGroup * 32 * 16 + 4096;   // = the single-split rows' place (never both)
 
   // ---- the end of a head's path, by all threads of a CTA (thread = output column): the appended token
   // joins as one more partial (level 0, weight 1, <q, k_new> in fp32), the ratio or the raw parts are
@@ -328,56 +341,69 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   struct NewTok {
     uint2 kn;                  // 4 dims of k_new per lane
     uint2 qv[kMaxGroup];       // 4 dims of q per lane and head (one head: slot 0)
-    float vn;                  // column tid of v_new
+    uint2 vn;                  // lanes 0-7: the columns 32 warp + 4 lane .. + 3 of v_new
     uint4 row_new;             // last warp: lanes 0-15 a piece of the row of K, lanes 16-31 of V
   };
   // h < 0: the queries of all heads
   auto load_new = [&](int h) -> NewTok {
     NewTok nt;
     nt.kn = make_uint2(0u, 0u);
-    nt.vn = 0.f;
+    nt.vn = make_uint2(0u, 0u);
     nt.row_new = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
     for (int k = 0; k < kMaxGroup; ++k) nt.qv[k] = make_uint2(0u, 0u);
     if (ap.k_new) {
-      nt.kn = *reinterpret_cast<const uint2*>(ap.k_new + (size_t)sl * kD + 4 * lane);
-      nt.vn = __bfloat162float(ap.v_new[(size_t)sl * kD + tid]);
+      nt.kn = ld_early_v2(ap.k_new + (size_t)sl * kD + 4 * lane);
+      if (lane < 8) nt.vn = ld_early_v2(ap.v_new + (size_t)sl * kD + 32 * warp + 4 * lane);
       const __nv_bfloat16* qs = q + ((size_t)seq * (G.H * g) + (size_t)head * g) * kD + 4 * lane;
       if (h >= 0) {
-        nt.qv[0] = *reinterpret_cast<const uint2*>(qs + (size_t)h * kD);
+        nt.qv[0] = ld_early_v2(qs + (size_t)h * kD);
       } else {
 #pragma unroll
         for (int k = 0; k < kMaxGroup; ++k)
-          if (k < g) nt.qv[k] = *reinterpret_cast<const uint2*>(qs + (size_t)k * kD);
+          if (k < g) nt.qv[k] = ld_early_v2(qs + (size_t)k * kD);
       }
       if (h <= 0 && warp == kWarps - 1)
-        nt.row_new = reinterpret_cast<const uint4*>((lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD)[lane & 15];
+        nt.row_new = ld_early_v4(reinterpret_cast<const uint4*>((lane < 16 ? ap.k_new : ap.v_new) + (size_t)sl * kD) + (lane & 15));
     }
     return nt;
   };
-  auto finish = [&](int h, float a, float M, float L, const NewTok& nt, int qslot) {
+  // base-2 logit of the appended token for the head whose query sits in slot qslot (by a whole warp)
+  auto score_new = [&](const NewTok& nt, int qslot) -> float {
+    const uint2 qv = nt.qv[qslot];
+    const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.y);
+    const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv.y);
+    float dot = __bfloat162float(q01.x) * __bfloat162float(k01.x);
+    dot = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), dot);
+    dot = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), dot);
+    dot = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), dot);
+    return warp_sum(dot) * sc;
+  };
+  // a: lanes 0-7 of every warp hold the sums of the output columns 32 warp + 4 lane .. + 3
+  auto finish = [&](int h, float4 a, float M, float L, const NewTok& nt, float x) {
     if (ap.k_new) {
-      const uint2 qv = nt.qv[qslot];
-      const __nv_bfloat162 k01 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.x), k23 = *reinterpret_cast<const __nv_bfloat162*>(&nt.kn.y);
-      const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qv.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qv.y);
-      float dot = __bfloat162float(q01.x) * __bfloat162float(k01.x);
-      dot = fmaf(__bfloat162float(q01.y), __bfloat162float(k01.y), dot);
-      dot = fmaf(__bfloat162float(q23.x), __bfloat162float(k23.x), dot);
-      dot = fmaf(__bfloat162float(q23.y), __bfloat162float(k23.y), dot);
-      const float x = warp_sum(dot) * sc;
       const float Mn = fmaxf(M, x);
       const float f = M == -INFINITY ? 0.f : fast_exp2(M - Mn), fN = fast_exp2(x - Mn);
-      a = fmaf(nt.vn, fN, a * f);
+      const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&nt.vn.x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&nt.vn.y);
+      a.x = fmaf(__bfloat162float(v01.x), fN, a.x * f); a.y = fmaf(__bfloat162float(v01.y), fN, a.y * f);
+      a.z = fmaf(__bfloat162float(v23.x), fN, a.z * f); a.w = fmaf(__bfloat162float(v23.y), fN, a.w * f);
       L = fmaf(L, f, fN);
       M = Mn;
     }
     const size_t qh = (size_t)seq * (G.H * g) + (size_t)head * g + h;
-    if (raw_acc) {
-      raw_acc[qh * kD + tid] = a;
-      if (tid == 0) { raw_ml[2 * qh] = M; raw_ml[2 * qh + 1] = L; }
-    } else {
-      const float inv = L > 0.f ? 1.0f / L : 0.f;
-      out[qh * kD + tid] = __float2bfloat16_rn(a * inv);
+    if (lane < 8) {
+      const int c = 32 * warp + 4 * lane;
+      if (raw_acc) {
+        *reinterpret_cast<float4*>(raw_acc + qh * kD + c) = a;
+        if (c == 0) { raw_ml[2 * qh] = M; raw_ml[2 * qh + 1] = L; }
+      } else {
+        const float inv = L > 0.f ? 1.0f / L : 0.f;
+        __nv_bfloat162 o01 = __floats2bfloat162_rn(a.x * inv, a.y * inv), o23 = __floats2bfloat162_rn(a.z * inv, a.w * inv);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t*>(&o01);
+        w.y = *reinterpret_cast<uint32_t*>(&o23);
+        *reinterpret_cast<uint2*>(out + qh * kD + c) = w;
+      }
     }
     if (ap.k_new && h == 0 && warp == kWarps - 1) {
       // append: one 256-byte row of K and of V, the position, the new length of C^0
@@ -402,20 +428,26 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       }
     }
   };
-  // Combine head h of this CTA's stream (all threads; thread = output column; see the combine below).
+  // Combine head h of this CTA's stream (see the combine below).  Warp w sums the columns 32 w .. 32 w + 31,
+  // a 128-byte line of every partial row: lane = (row group rg = lane / 8, 16-byte piece lane % 8), the lane
+  // takes the rows rg, rg + 4, ... (vector loads and stores: a quarter of the memory instructions that a
+  // lane per column would need), and the four row groups meet by two shuffle steps.
   auto combine_head = [&](int h) {
-    const float* rows = part + ((size_t)sl * splits * g + h) * kD + tid;                         // row of split sp: + sp rstep
-    const float* mls = part + (size_t)gridDim.x * splits * g * kD + ((size_t)sl * splits * g + h) * 2;   // its pair: + sp g 2
-    const size_t rstep = (size_t)g * kD;
+    const int rg = lane >> 3;
+    const float* rows = part + ((size_t)sl * splits * g + h) * kD + 32 * warp + 4 * (lane & 7);        // row of split sp: + sp rstep
+    const float* mls = part + (size_t)gridDim.x * splits * g * kD + (((size_t)sl * splits * g + h) * kWarps + warp) * 2;   // this warp's copy of its pair: + sp mstep
+    const size_t rstep = (size_t)g * kD, mstep = (size_t)g * kWarps * 2;
     const NewTok nt = load_new(h);              // in flight during the polls
-    const float* mlp[2] = {mls + (size_t)lane * g * 2, mls + (size_t)(lane + 32) * g * 2};
+    const float* mlp[2] = {mls + (size_t)lane * mstep, mls + (size_t)(lane + 32) * mstep};
     float2 ml[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) ml[e] = lane + 32 * e < splits ? ld_poll2(mlp[e]) : make_float2(-INFINITY, 0.f);
-    float v[kMaxSplits];
+    constexpr int kPer = kMaxSplits / 4;
+    float4 v[kPer];
 #pragma unroll
-    for (int j = 0; j < kMaxSplits; ++j)
-      if (j < splits) v[j] = ld_poll1(rows + j * rstep);
+    for (int i = 0; i < kPer; ++i)
+      if (rg + 4 * i < splits) v[i] = ld_poll4(rows + (size_t)(rg + 4 * i) * rstep);
+    const float x_new = ap.k_new ? score_new(nt, 0) : 0.f;      // while the polls are in flight
     // A round re-reads everything that was still empty, all loads in flight together (words checked one
     // after the other would cost a round trip each).
     const long long t0 = clock64();
@@ -429,9 +461,9 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
           pending = true;
         }
 #pragma unroll
-      for (int j = 0; j < kMaxSplits; ++j)
-        if (j < splits && is_empty(v[j])) {
-          v[j] = ld_poll1(rows + j * rstep);
+      for (int i = 0; i < kPer; ++i)
+        if (rg + 4 * i < splits && (is_empty(v[i].x) || is_empty(v[i].y) || is_empty(v[i].z) || is_empty(v[i].w))) {
+          v[i] = ld_poll4(rows + (size_t)(rg + 4 * i) * rstep);
           pending = true;
         }
       if (!pending) break;
@@ -442,18 +474,32 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     const float f0 = ml[0].x == -INFINITY ? 0.f : fast_exp2(ml[0].x - M);
     const float f1 = ml[1].x == -INFINITY ? 0.f : fast_exp2(ml[1].x - M);
     const float L = warp_sum(fmaf(ml[0].y, f0, ml[1].y * f1));
-    float a = 0.f;
+    // the factors of all splits through shared memory (behind the merge buffers, which other warps of the
+    // last split's CTA may still be reading)
+    float* fac = reinterpret_cast<float*>(tiles + kFacOff) + warp * kMaxSplits;
+    fac[lane] = f0;
+    fac[lane + 32] = f1;
+    __syncwarp();
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < kMaxSplits; ++j)
-      if (j < splits) a = fmaf(v[j], __shfl_sync(0xffffffffu, j < 32 ? f0 : f1, j & 31), a);
-    finish(h, a, M, L, nt, 0);
-    // the empty pattern again, for the next launch (the pairs once every warp has read them)
-    const float e = __uint_as_float(kEmptyWord);
+    for (int i = 0; i < kPer; ++i)
+      if (rg + 4 * i < splits) {
+        const float f = fac[rg + 4 * i];
+        a.x = fmaf(v[i].x, f, a.x); a.y = fmaf(v[i].y, f, a.y); a.z = fmaf(v[i].z, f, a.z); a.w = fmaf(v[i].w, f, a.w);
+      }
 #pragma unroll
-    for (int j = 0; j < kMaxSplits; ++j)
-      if (j < splits) __stcg(const_cast<float*>(rows + j * rstep), e);
-    __syncthreads();
-    if (warp == 0) {
+    for (int o = 8; o < 32; o <<= 1) {
+      a.x += __shfl_xor_sync(0xffffffffu, a.x, o); a.y += __shfl_xor_sync(0xffffffffu, a.y, o);
+      a.z += __shfl_xor_sync(0xffffffffu, a.z, o); a.w += __shfl_xor_sync(0xffffffffu, a.w, o);
+    }
+    finish(h, a, M, L, nt, x_new);
+    // the empty pattern again, for the next launch (every warp has its own copy of the pairs, so nobody else
+    // still wants these words)
+    {
+      const float e = __uint_as_float(kEmptyWord);
+#pragma unroll
+      for (int i = 0; i < kPer; ++i)
+        if (rg + 4 * i < splits) __stcg(reinterpret_cast<float4*>(const_cast<float*>(rows + (size_t)(rg + 4 * i) * rstep)), make_float4(e, e, e, e));
 #pragma unroll
       for (int k = 0; k < 2; ++k)
         if (lane + 32 * k < splits) __stcg(reinterpret_cast<float2*>(const_cast<float*>(mlp[k])), make_float2(e, e));
@@ -633,7 +679,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const size_t n_rows_all = (size_t)gridDim.x * splits * g;
   float* my_acc = single ? reinterpret_cast<float*>(tiles + kSingleOff) : part + ((size_t)sl * splits + split) * g * kD;
   float* my_ml = single ? reinterpret_cast<float*>(tiles + kSingleOff) + kMaxGroup * kD
-                        : part + n_rows_all * kD + ((size_t)sl * splits + split) * g * 2;
+                        : part + n_rows_all * kD + ((size_t)sl * splits + split) * g * 2 * kWarps;
   // Work items of the merge and combine phases: (head mh, way mw), item r = mw g + mh, ways =
   // max(1, warps / g); a warp takes items r = warp, warp + kWarps, ... (lane = 4 output columns).
   // The ways of a head share its rows: way mw takes the rows mw, mw + ways, ...
@@ -690,7 +736,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
       } else {                                  // published: see the combine below
         __stcg(reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane), acc);
-        if (lane == 0) __stcg(reinterpret_cast<float2*>(my_ml + 2 * h), make_float2(M, L));
+        if (lane < kWarps) __stcg(reinterpret_cast<float2*>(my_ml + (h * kWarps + lane) * 2), make_float2(M, L));   // a copy per combining warp
       }
     }
   }
@@ -710,7 +756,9 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
     NewTok nt = load_new(-1);
 #pragma unroll
     for (int h = 0; h < kMaxGroup; ++h)
-      if (h < g) finish(h, acc1[h * kD + tid], ml1[2 * h], ml1[2 * h + 1], nt, h);
+      if (h < g)
+        finish(h, *reinterpret_cast<const float4*>(acc1 + h * kD + 32 * warp + 4 * (lane & 7)), ml1[2 * h], ml1[2 * h + 1], nt,
+               ap.k_new ? score_new(nt, h) : 0.f);
     return;
   }
   if (split == splits - 1) combine_head(0);
