@@ -112,6 +112,8 @@ __device__ inline float fast_exp2(float x) {     // -inf -> 0
 // Polling loads of the split-K scratch (see the combine): never served by L1.
 constexpr uint32_t kEmptyWord = 0xffffffffu;
 constexpr int kMaxSplits = 64;
+static_assert(2 * kWarps <= 8, "the scratch holds 8 floats of (max, sum) copies per partial row (decode_scratch_bytes)");
+static_assert(kThreads == kD, "the combine maps a warp to 32 output columns");
 __device__ inline bool is_empty(float x) { return __float_as_uint(x) == kEmptyWord; }
 // Plain loads as volatile asm statements: they keep their place among the polling loads, i.e. they are issued
 // before the polls and not where their values are first used.
@@ -516,13 +518,18 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   // one mma.sync.m16n8k16 per 16 tokens x 16 dims instead of the two that a query-major tile
   // (16 rows, at most 8 of them used) needs.
   const int hq = lane >> 2, tq = lane & 3;         // C fragment: rows hq, hq + 8; columns 2 tq, 2 tq + 1
+  // With g <= 4 the columns 4-7 of the operand repeat the heads 0-3: both halves compute the same scores, and
+  // in the second product the columns 0-3 carry the high parts of the probabilities and the columns 4-7 their
+  // low parts, so that one MMA does what takes two with more heads; the halves are added before the merge.
+  const bool packed = g <= 4;
   uint32_t qb[8][2];
   {
-    const __nv_bfloat16* qp = q + ((size_t)seq * (G.H * g) + (size_t)head * g + hq) * kD;
+    const int hr = packed ? hq & 3 : hq;
+    const __nv_bfloat16* qp = q + ((size_t)seq * (G.H * g) + (size_t)head * g + hr) * kD;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       uint32_t lo = 0, hi = 0;
-      if (hq < g) {
+      if (hr < g) {
         lo = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 2 * tq);
         hi = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * tq);
       }
@@ -629,18 +636,30 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         const uint32_t ph0 = pack_bf16(x[tb][0], x[tb][1]), ph1 = pack_bf16(x[tb][2], x[tb][3]);
         const uint32_t pl0 = pack_bf16(x[tb][0] - bf16_lo(ph0), x[tb][1] - bf16_hi(ph0));
         const uint32_t pl1 = pack_bf16(x[tb][2] - bf16_lo(ph1), x[tb][3] - bf16_hi(ph1));
-        bh[tb][0] = movm_trans(ph0); bh[tb][1] = movm_trans(ph1);
-        bl[tb][0] = movm_trans(pl0); bl[tb][1] = movm_trans(pl1);
+        if (packed) {                          // this thread's two columns: high parts (tq < 2) or low parts
+          bh[tb][0] = movm_trans(tq < 2 ? ph0 : pl0); bh[tb][1] = movm_trans(tq < 2 ? ph1 : pl1);
+          bl[tb][0] = bl[tb][1] = 0u;
+        } else {
+          bh[tb][0] = movm_trans(ph0); bh[tb][1] = movm_trans(ph1);
+          bl[tb][0] = movm_trans(pl0); bl[tb][1] = movm_trans(pl1);
+        }
       }
       // ---- O^T[128 x 8] += V^T[128 x 16 kTB] P^T[16 kTB x 8]: the high parts of a block, then its low
       // parts, so that no MMA follows its predecessor on the same accumulator
       if (!keys_only) {
+        if (packed) {
 #pragma unroll
-        for (int tb = 0; tb < kTB; ++tb) {
+          for (int tb = 0; tb < kTB; ++tb)
 #pragma unroll
-          for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bh[tb][0], bh[tb][1]);
+            for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bh[tb][0], bh[tb][1]);
+        } else {
 #pragma unroll
-          for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bl[tb][0], bl[tb][1]);
+          for (int tb = 0; tb < kTB; ++tb) {
+#pragma unroll
+            for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bh[tb][0], bh[tb][1]);
+#pragma unroll
+            for (int mb = 0; mb < 8; ++mb) mma_bf16(o[mb], va[tb][mb], bl[tb][0], bl[tb][1]);
+          }
         }
       }
     }
@@ -656,6 +675,12 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   for (int off = 4; off < 32; off <<= 1) {
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+  }
+  if (packed) {                                // high + low halves: the columns 2 tq + e and 2 tq + e + 4
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[n][j] += __shfl_xor_sync(0xffffffffu, o[n][j], 2);
   }
   __syncthreads();
 #pragma unroll
