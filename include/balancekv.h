@@ -168,7 +168,7 @@ int balancekv_decode_attn_host(balancekv_ctx* ctx, int layer, const void* q_host
  * that loads the library, until the process exits); the call performs no cudaMalloc, cudaFree
  * or other allocating call.  A problem whose scratch (256 bytes, a segment table of
  * n_streams * (level+1) * 8 bytes, n_streams ticket words rounded up to 64, and n_streams *
- * splits * group * (head_dim+4) * 4 bytes of partial rows, splits <= 64 chosen from the SM
+ * splits * group * (head_dim+8) * 4 bytes of partial rows, splits <= 64 chosen from the SM
  * count) exceeds the array is rejected with BALANCEKV_E_NOMEM and a message on stderr.  The
  * first call on a device -- of this function or of balancekv_decode_attn_static_status,
  * whichever host thread gets there first -- looks up the array's device address

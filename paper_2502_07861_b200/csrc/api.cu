@@ -133,7 +133,7 @@ struct balancekv_ctx {
   // two-instance estimator: un-normalised parts of the numerator and denominator instances, unit values
   float* two_acc = nullptr;             // [BALANCEKV_MAX_MERGE][B, Hq, d] value sums per merged slot
   float* two_ml = nullptr;              // [BALANCEKV_MAX_MERGE][B, Hq, 2] (max, sum) per merged slot
-  float* two_scratch = nullptr;         // [BALANCEKV_MAX_MERGE] split-K scratch blocks (tickets + partial rows)
+  float* two_scratch = nullptr;         // [BALANCEKV_MAX_MERGE] split-K scratch blocks (laid out like d_decode_scratch)
   size_t two_scratch_words = 0;         // 4-byte words per block
   void* unit_V = nullptr;               // rows (1, 0, ..., 0) for balancekv_stream_append_layer_keys
   size_t unit_rows = 0;

@@ -8,18 +8,19 @@
 // at g = 5 the CUDA-core formulation needs ~65 instructions per token and is issue bound far below
 // HBM speed, this one needs ~3.
 //
-// Grid (streams of the layer, splits), one CTA of 16 warps in eight groups per SM.  A CTA walks its share of the stream's
-// 64-token tiles through a 6-stage ring filled by TMA (tensor maps over the K and V arenas, boxes of
-// 64 dims x 64 rows, 128-byte swizzle, so ldmatrix reads are bank-conflict free); the groups take
-// tiles in turn.  Warp w of a group owns tokens 32w..32w+31 of a tile -- the tokens are the M
-// dimension of both products -- and keeps a private online softmax (running max, sum, 128 x 8
-// accumulator) in registers; warps merge through shared memory, splits through a global scratch
-// and a ticket counter (the last CTA of a stream combines; nobody waits).
+// Grid (streams of the layer, splits [+ g - 1], slots), CTAs of four warps in two groups, two per SM.  A CTA
+// walks its share of the stream's 64-token tiles through a 3-stage ring filled by TMA (tensor maps over the K
+// and V arenas, boxes of 64 dims x 64 rows, 128-byte swizzle, so ldmatrix reads are bank-conflict free); the
+// groups take tiles in turn.  Warp w of a group owns tokens 32w..32w+31 of a tile -- the tokens are the M
+// dimension of both products -- and keeps a private online softmax (running max, sum, 128 x 8 accumulator)
+// in registers; warps merge through shared memory, splits through a global scratch whose words are their own
+// arrival flags: with more than one split, head 0 of a stream is combined by the CTA of its last split and
+// head h > 0 by a CTA of its own (grid y = splits + h - 1), which polls the partial rows of its head.
 // Fused decode step: with k_new / v_new given, the launch also appends one token per stream
-// (Algorithm 3's C^0 <- C^0 + {(k_j, v_j)}).  The new token never goes through the tiles: the
-// combining CTA scores it in fp32, adds it as one more partial (weight 1) and only then writes
-// its row, its position and the stream's new level-0 length, after every CTA of the stream has
-// taken its ticket, i.e. has finished reading the old segment table.
+// (Algorithm 3's C^0 <- C^0 + {(k_j, v_j)}).  The new token never goes through the tiles: the combining
+// CTAs score it in fp32 and add it as one more partial (weight 1), and the combiner of head 0 writes its
+// row, its position and the stream's new level-0 length once its polls have shown that every CTA of the
+// stream is past its tiles, i.e. has finished reading the old segment table.
 // Rows of a tile beyond a segment's end are masked in the scores; their V rows are whatever the
 // arena holds there (zero-initialised at creation or finite older rows) times an exact zero.
 #include <cuda.h>
@@ -695,7 +696,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   }
   __syncthreads();
   // With a single split the CTA's partial is the stream's result: it stays in shared memory (behind
-  // the merge buffers) and the ticket, the fences and the staging copy are skipped.
+  // the merge buffers) and goes straight to the end of the heads' path.
   constexpr uint32_t kMrg2Off = kWarps * kMaxGroup * PS * 4;        // behind mrg: [ways][g][PS] first-level merges
   constexpr uint32_t kSingleOff = 4352 + kWarps * kMaxGroup * 32 * 16 + 4096;   // behind the merge buffers and the combine's tables
   const bool single = splits == 1;
@@ -840,8 +841,8 @@ cudaError_t launch_decode_step_mma(const Geom& G, const Arena& A, int layer, con
                                    int rel_row, int idx0, int new_len, const Seg* seg_hint, int early, const int* in_flag,
                                    int in_expect, cudaStream_t st);
 
-// Scratch layout of all launches: ticket counters, then (stream, split, head) rows of kD column sums,
-// then their (max, sum) pairs.
+// Scratch layout of all launches: the CUDA-core kernel's ticket counters (unused here), then (stream, split,
+// head) rows of kD column sums, then per row kWarps copies of its (max, sum) pair.
 // Un-normalised parts (see StepAppend::raw_acc) of the layer's streams, for decode merged over slots.
 cudaError_t launch_decode_parts_mma(const Geom& G, const Arena& A, int layer, const void* q, float* raw_acc, float* raw_ml,
                                     float* scratch, int splits, int* status, const void* maps, int keys_only,
