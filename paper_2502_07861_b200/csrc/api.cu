@@ -314,9 +314,13 @@ int balancekv_create(const balancekv_config* cfg, balancekv_ctx** out) {
   const size_t row_bytes = (size_t)f.head_dim * c->esz;
   if (T > 0) {
     const size_t per_call = (size_t)(t / 2) * row_bytes * 2;          // K+V survivors of one call
-    const size_t budget = (size_t)256 << 20;                          // both pools together
+    // Both pools together: up to 1 GiB, so that a batched launch spans many waves of CTAs (a launch of
+    // 256 calls is 1.7 waves on 148 SMs: 86 % of its slots), but no more than the level-0 calls that can
+    // be pending at once.
+    const size_t budget = (size_t)1 << 30;
     int64_t mc = (int64_t)(budget / (2 * per_call));
-    mc = std::max<int64_t>(2, std::min<int64_t>(mc, 4096));
+    const int64_t pending_calls = (int64_t)c->n_streams * ((max_pending + t - 1) / t);
+    mc = std::max<int64_t>(2, std::min<int64_t>(std::min<int64_t>(mc, pending_calls), 4096));
     c->max_calls = (int)mc;
     c->Lo.pool_pairs = T > 1 ? (mc + 1) / 2 : 0;
   }
