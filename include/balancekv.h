@@ -318,6 +318,13 @@ int balancekv_profile_read(balancekv_ctx* ctx, double* out_host);
  * kernel whose bounded wait ran out would.  Synchronises the device. */
 int balancekv_debug_set_status(balancekv_ctx* ctx, int value);
 
+/* Testing aid: the number of 4-byte words of the split-K decode scratch that do not hold the
+ * "empty" pattern (Algorithm 1's output ratio is summed over splits through that scratch; the
+ * tensor-core decode kernel uses each word as its own arrival flag and must leave every word
+ * empty behind every launch).  0 for contexts on the CUDA-core decode kernel.  Synchronises the
+ * device.  words: host pointer. */
+int balancekv_debug_scratch_used(balancekv_ctx* ctx, int64_t* words);
+
 /* Synchronises the device.  Returns BALANCEKV_E_TIMEOUT (record filled) if a device-side wait gave up. */
 int balancekv_stats(balancekv_ctx* ctx, balancekv_stats_t* out);
 const char* balancekv_strerror(int code);

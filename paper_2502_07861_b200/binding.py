@@ -24,7 +24,7 @@ EXPORTS = [
     "balancekv_profile_enable", "balancekv_profile_sample", "balancekv_profile_read", "balancekv_decode_attn_static",
     "balancekv_stream_step", "balancekv_stream_step_host", "balancekv_stream_append_layer_keys",
     "balancekv_decode_attn_two", "balancekv_decode_attn_merged", "balancekv_stream_append_bucketed",
-    "balancekv_stream_append_layer_bucketed", "balancekv_stream_append_layer_preserving", "balancekv_debug_set_status", "balancekv_decode_attn_static_status",
+    "balancekv_stream_append_layer_bucketed", "balancekv_stream_append_layer_preserving", "balancekv_debug_set_status", "balancekv_decode_attn_static_status", "balancekv_debug_scratch_used",
 ]
 PROFILE_CLASSES = ("append", "radii", "gram_walk", "compact", "decode", "bookkeeping")
 
@@ -99,6 +99,7 @@ def load():
     lib.balancekv_decode_attn_static.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, ci, ci, ci, vp]
     lib.balancekv_decode_attn_static_status.argtypes = [vp, vp]
     lib.balancekv_debug_set_status.argtypes = [vp, ci]
+    lib.balancekv_debug_scratch_used.argtypes = [vp, C.POINTER(C.c_int64)]
     for name in EXPORTS:
         if name != "balancekv_strerror":
             getattr(lib, name).restype = ci
@@ -361,6 +362,12 @@ class Context:
         torch.cuda.synchronize()
         return (_from_ptr(pe.value, (m.value,), torch.int8), _from_ptr(ps.value, (m.value,), torch.float32),
                 _from_ptr(pp.value, (m.value,), torch.float32))
+
+    def debug_scratch_used(self) -> int:
+        """Words of the split-K decode scratch that are not empty (0 between launches)."""
+        n = C.c_int64(0)
+        _check(self.lib.balancekv_debug_scratch_used(self._h, C.byref(n)), "balancekv_debug_scratch_used")
+        return int(n.value)
 
     def debug_set_status(self, value):
         """Testing aid: overwrite the device status word (1 = a bounded wait gave up)."""

@@ -1371,6 +1371,26 @@ int balancekv_debug_set_status(balancekv_ctx* c, int value) {
   return BALANCEKV_OK;
 }
 
+int balancekv_debug_scratch_used(balancekv_ctx* c, int64_t* words) {
+  if (!c || !words) return BALANCEKV_E_INVAL;
+  *words = 0;
+  if (!c->decode_maps) return BALANCEKV_OK;          // the CUDA-core kernel keeps no state in its partial rows
+  BKV_CUDA(cudaDeviceSynchronize());
+  const size_t n_sl = (size_t)c->G.B * c->G.H;
+  const size_t ticket_words = ((n_sl + 63) / 64) * 64;
+  auto count = [&](const float* block, size_t bytes) -> int {
+    std::vector<uint32_t> host(bytes / 4);
+    if (cudaMemcpy(host.data(), block, host.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BALANCEKV_E_CUDA;
+    for (size_t i = ticket_words; i < host.size(); ++i) *words += host[i] != 0xffffffffu;
+    return BALANCEKV_OK;
+  };
+  int rc = count(c->d_decode_scratch, decode_scratch_bytes(c->G, c->max_splits));
+  if (rc == BALANCEKV_OK && c->two_scratch)
+    for (int z = 0; z < BALANCEKV_MAX_MERGE && rc == BALANCEKV_OK; ++z)
+      rc = count(c->two_scratch + c->two_scratch_words * z, c->two_scratch_words * 4);
+  return rc;
+}
+
 int balancekv_plan_calls(int block, int levels, int recent_window, const int32_t* appended_after_event, int n_events,
                          int32_t* calls_out, int max_calls) {
   if (block < 2 || block % 2 || levels < 0 || levels > kMaxLevels || recent_window < 0 || !appended_after_event ||

@@ -294,10 +294,11 @@ def test_a_timed_out_wait_surfaces_as_an_error_code_and_reset_clears_it(cuda_lib
 @pytest.mark.parametrize("g", [1, 2, 3, 5, 6, 7, 8])
 @pytest.mark.parametrize("splits", [1, 5, 24, 64])
 def test_decode_kernel_every_group_size_and_split_factor(cuda_lib, g, splits):
-    """The tensor-core decode kernel against the oracle's weighted attention for every group size and for split
-    factors that take each of its combine paths: a single split (no ticket), partial rows staged in shared memory,
-    and more partial rows than fit there (read from global memory: g = 8 with 24 or 64 splits).  Two levels with
-    ragged lengths, one of them shorter than a tile."""
+    """The tensor-core decode kernel against the oracle's weighted attention for every group size (g <= 4 packs the
+    high and low parts of the probabilities into one MMA) and for split factors that take each of its combine
+    paths: a single split (the result stays in the CTA), a few splits, more splits than tiles (empty partial rows),
+    and a grid of several waves (64 splits + g - 1 combining CTAs per stream).  Two levels with ragged lengths, one
+    of them shorter than a tile.  Behind every launch the split-K scratch is empty again."""
     B, H, d, T, n_heavy, n_tail = 1, 2, 128, 2, 2500, 37
     ctx = cuda_lib.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=64, levels=T,
                            max_tokens=(n_heavy << T) + 64, decode_splits=splits)
@@ -305,12 +306,49 @@ def test_decode_kernel_every_group_size_and_split_factor(cuda_lib, g, splits):
     ctx.cache_load_level(0, T, to_device(K[:, :, :n_heavy], "bf16"), to_device(V[:, :, :n_heavy], "bf16"))
     ctx.stream_append_layer(0, to_device(K[:, :, n_heavy:], "bf16"), to_device(V[:, :, n_heavy:], "bf16"))
     w = np.concatenate([np.full(n_heavy, 4.0), np.ones(n_tail)])
-    for step in range(2):                                   # twice: the tickets and the scratch are reused
+    for step in range(2):                                   # twice: the scratch is reused
         q = synth.queries(31, 0, step, B, H * g, d, "bf16")
         out = ctx.decode_attn(0, to_device(q, "bf16")).float().cpu().numpy()
+        assert ctx.debug_scratch_used() == 0
         for h in range(H):
             ref = oracle.weighted_attention(K[0, h], V[0, h], w, q[0, h * g:(h + 1) * g])
             assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3, (g, splits, h)
+    st = ctx.stats()
+    assert st["device_status"] == 0 and st["decode_kernel"] == 2
+    ctx.close()
+
+
+def test_decode_scratch_is_empty_behind_every_launch_while_the_split_factor_moves(cuda_lib):
+    """The partial rows of the tensor-core decode kernel are their own arrival flags: a launch must find and leave
+    every word of the split-K scratch empty, whatever split factor the launch before it used.  Decode steps (attend +
+    append) with compress points in between walk the automatic split factor through several values; every output is
+    checked against the oracle's weighted attention over the library's own cache view."""
+    B, H, g, d, t, T = 1, 2, 4, 128, 64, 2
+    ctx = cuda_lib.Context(n_seqs=B, n_layers=1, n_kv_heads=H, n_q_heads=H * g, head_dim=d, dtype="bf16", block=t, levels=T,
+                           max_tokens=8192)
+    K, V = synth.layer_kv("llama", 77, 0, B, H, 6000, d, "bf16")
+    pos = 0
+    for n_new in (130, 700, 64, 2100, 1500):
+        ctx.stream_append_layer(0, to_device(K[:, :, pos:pos + n_new], "bf16"), to_device(V[:, :, pos:pos + n_new], "bf16"))
+        pos += n_new
+        ctx.compress()
+        for step in range(3):
+            q = synth.queries(77, 0, pos + step, B, H * g, d, "bf16")
+            kn, vn = K[:, :, pos], V[:, :, pos]                                  # [B, H, d]
+            views = [ctx.cache_view(0, 0, h) for h in range(H)]                  # the weighted set before the step
+            q_t = to_device(q, "bf16")
+            out_t = q_t.clone()
+            ctx.stream_step(0, q_t, to_device(kn, "bf16"), to_device(vn, "bf16"), out_t)
+            out = out_t.float().cpu().numpy()
+            pos += 1
+            assert ctx.debug_scratch_used() == 0
+            for h in range(H):
+                vK, vV, vw, _ = views[h]
+                Kh = np.concatenate([vK.float().cpu().numpy().astype(np.float64), kn[0, h][None].astype(np.float64)])
+                Vh = np.concatenate([vV.float().cpu().numpy().astype(np.float64), vn[0, h][None].astype(np.float64)])
+                wh = np.concatenate([vw.float().cpu().numpy().astype(np.float64), np.ones(1)])
+                ref = oracle.weighted_attention(Kh, Vh, wh, q[0, h * g:(h + 1) * g])
+                assert rel_l2(out[0, h * g:(h + 1) * g], ref) <= 2e-3, (pos, h, len(wh))
     st = ctx.stats()
     assert st["device_status"] == 0 and st["decode_kernel"] == 2
     ctx.close()
