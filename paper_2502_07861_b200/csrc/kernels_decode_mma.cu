@@ -438,8 +438,8 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   auto combine_head = [&](int h) {
     const int rg = lane >> 3;
     const float* rows = part + ((size_t)sl * splits * g + h) * kD + 32 * warp + 4 * (lane & 7);        // row of split sp: + sp rstep
-    const float* mls = part + (size_t)gridDim.x * splits * g * kD + (((size_t)sl * splits * g + h) * kWarps + warp) * 2;   // this warp's copy of its pair: + sp mstep
-    const size_t rstep = (size_t)g * kD, mstep = (size_t)g * kWarps * 2;
+    const float* mls = part + (size_t)gridDim.x * splits * g * kD + (((size_t)sl * g + h) * kWarps + warp) * splits * 2;   // this warp's copies of the head's pairs, split by split: one line or two for a polling warp
+    const size_t rstep = (size_t)g * kD, mstep = 2;
     const NewTok nt = load_new(h);              // in flight during the polls
     const float* mlp[2] = {mls + (size_t)lane * mstep, mls + (size_t)(lane + 32) * mstep};
     float2 ml[2];
@@ -705,7 +705,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
   const size_t n_rows_all = (size_t)gridDim.x * splits * g;
   float* my_acc = single ? reinterpret_cast<float*>(tiles + kSingleOff) : part + ((size_t)sl * splits + split) * g * kD;
   float* my_ml = single ? reinterpret_cast<float*>(tiles + kSingleOff) + kMaxGroup * kD
-                        : part + n_rows_all * kD + ((size_t)sl * splits + split) * g * 2 * kWarps;
+                        : part + n_rows_all * kD + (size_t)sl * g * kWarps * splits * 2;       // pair of (head, copy, split): + ((h kWarps + copy) splits + split) 2
   // Work items of the merge and combine phases: (head mh, way mw), item r = mw g + mh, ways =
   // max(1, warps / g); a warp takes items r = warp, warp + kWarps, ... (lane = 4 output columns).
   // The ways of a head share its rows: way mw takes the rows mw, mw + ways, ...
@@ -762,7 +762,7 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
       } else {                                  // published: see the combine below
         __stcg(reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane), acc);
-        if (lane < kWarps) __stcg(reinterpret_cast<float2*>(my_ml + (h * kWarps + lane) * 2), make_float2(M, L));   // a copy per combining warp
+        if (lane < kWarps) __stcg(reinterpret_cast<float2*>(my_ml + ((size_t)(h * kWarps + lane) * splits + split) * 2), make_float2(M, L));   // a copy per combining warp
       }
     }
   }
