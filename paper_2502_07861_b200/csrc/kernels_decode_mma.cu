@@ -110,7 +110,8 @@ __device__ inline float fast_exp2(float x) {     // -inf -> 0
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Polling loads of the split-K scratch (see the combine): never served by L1.
+// Accesses to the split-K scratch (see the combine).  Publishing stores and polling loads are relaxed operations at
+// GPU scope -- never served by L1, and not a data race although nothing else orders them: each word validates itself.
 constexpr uint32_t kEmptyWord = 0xffffffffu;
 constexpr int kMaxSplits = 64;
 static_assert(2 * kWarps <= 8, "the scratch holds 8 floats of (max, sum) copies per partial row (decode_scratch_bytes)");
@@ -130,13 +131,19 @@ __device__ inline uint4 ld_early_v4(const void* p) {
 }
 __device__ inline float4 ld_poll4(const float* p) {
   float4 v;
-  asm volatile("ld.volatile.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
   return v;
 }
 __device__ inline float2 ld_poll2(const float* p) {
   float2 v;
-  asm volatile("ld.volatile.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
   return v;
+}
+__device__ inline void st_scratch4(float* p, float4 v) {
+  asm volatile("st.relaxed.gpu.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ inline void st_scratch2(float* p, float2 v) {
+  asm volatile("st.relaxed.gpu.global.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(v.x), "f"(v.y) : "memory");
 }
 __device__ inline uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -502,10 +509,10 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
       const float e = __uint_as_float(kEmptyWord);
 #pragma unroll
       for (int i = 0; i < kPer; ++i)
-        if (rg + 4 * i < splits) __stcg(reinterpret_cast<float4*>(const_cast<float*>(rows + (size_t)(rg + 4 * i) * rstep)), make_float4(e, e, e, e));
+        if (rg + 4 * i < splits) st_scratch4(const_cast<float*>(rows + (size_t)(rg + 4 * i) * rstep), make_float4(e, e, e, e));
 #pragma unroll
       for (int k = 0; k < 2; ++k)
-        if (lane + 32 * k < splits) __stcg(reinterpret_cast<float2*>(const_cast<float*>(mlp[k])), make_float2(e, e));
+        if (lane + 32 * k < splits) st_scratch2(const_cast<float*>(mlp[k]), make_float2(e, e));
     }
     if (!ok && lane == 0) atomicCAS(status, kStatusOk, kStatusWaitTimeout);
   };
@@ -761,14 +768,14 @@ decode_mma_kernel(Geom G, Arena A, int layer, const __nv_bfloat16* __restrict__ 
         *reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane) = acc;
         if (lane == 0) *reinterpret_cast<float2*>(my_ml + 2 * h) = make_float2(M, L);
       } else {                                  // published: see the combine below
-        __stcg(reinterpret_cast<float4*>(my_acc + h * kD + 4 * lane), acc);
-        if (lane < kWarps) __stcg(reinterpret_cast<float2*>(my_ml + ((size_t)(h * kWarps + lane) * splits + split) * 2), make_float2(M, L));   // a copy per combining warp
+        st_scratch4(my_acc + h * kD + 4 * lane, acc);
+        if (lane < kWarps) st_scratch2(my_ml + ((size_t)(h * kWarps + lane) * splits + split) * 2, make_float2(M, L));   // a copy per combining warp
       }
     }
   }
   // ---- combine.  No ticket, no fence and no staging copy: a word of the scratch is its own arrival flag.
   // Between launches every word of the partial rows holds kEmptyWord, a NaN pattern that arithmetic never
-  // produces (results are canonical NaNs, and -inf is a legal maximum).  A CTA publishes its rows with plain
+  // produces (results are canonical NaNs, and -inf is a legal maximum).  A CTA publishes its rows with relaxed
   // stores.  Head 0 of a stream is combined by the stream's CTA of the last split, head h > 0 by the CTA
   // (stream, splits + h - 1), which has no tiles: the g combiners of a stream run side by side on different
   // SMs, each polls the words of its head until none is empty, sums, and puts the empty pattern back for the
